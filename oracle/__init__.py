@@ -1,0 +1,16 @@
+"""CPU oracle for streamlined few-bit QNN inference -- TEST INFRASTRUCTURE ONLY.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import
+this package.  It shares no code with the CUDA path and never imports it.
+
+Contents
+--------
+qnn_oracle.c   plain C loops: integer GEMM, thresholding, direct convolution,
+               max-pool (compiled by ``oracle.build``).
+oracle.py      ctypes access to the C functions on numpy arrays.
+bitserial.py   Algorithms 1 and 2 of the paper restated on Python integers
+               (tiny sizes only; used to pin the GEMM oracle).
+streamline.py  float batch-norm + quantizer reference and the threshold
+               absorption of Section 2.1 (fp64).
+alexnet.py     the AlexNet-shaped layer chain of Section 4.2 built from the above.
+"""
