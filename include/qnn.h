@@ -1,0 +1,207 @@
+/*
+ * qnn.h -- C ABI of the B200 (sm_100a) hot path of streamlined few-bit QNN
+ * inference: few-bit integer GEMM WwAa fused with the per-output-channel
+ * multi-threshold activation, fed by channel-interleaved lowering.
+ *
+ * General conventions
+ * -------------------
+ *  - Shapes follow the paper's (rows, depth, cols) = (M, K, N) of Section 4.1:
+ *    M output channels (weight rows), K depth, N columns (pixels x batch).
+ *    Both operands are indexed (row-or-column, depth) as in Algorithm 1, i.e.
+ *    the activation matrix is held transposed: W is [M][K], A is [N][K].
+ *  - Every data pointer is a DEVICE pointer owned by the caller; descriptors
+ *    are host structs read during the call.  The library allocates no device
+ *    memory: scratch is sized by a *_workspace_bytes query and passed in.
+ *  - `stream` is a cudaStream_t passed as void*.  Calls only enqueue work on
+ *    that stream; they never synchronise (the two functions that return a
+ *    value read back from the device say so).
+ *  - Errors are return codes.  Argument errors are detected on the host before
+ *    anything is launched.  Device code never traps: a bounded wait that runs
+ *    out records QNN_ERR_DEVICE_TIMEOUT in a device status word that
+ *    qnn_device_status() reads.
+ *  - All results are exact integers; there is no CPU fallback and no other
+ *    backend.
+ *
+ * Encodings (Section 3.1; the paper's Algorithm 2 is the SIGNED x SIGNED case)
+ *   QNN_ENC_UNSIGNED  b bits, value in [0, 2^b - 1]
+ *   QNN_ENC_SIGNED    b bits two's complement, value in [-2^(b-1), 2^(b-1)-1]
+ *   QNN_ENC_BIPOLAR   1 bit, bit 1 -> +1, bit 0 -> -1
+ *
+ * Operand formats
+ *   QNN_FMT_BITPLANES  uint32 [bits][rows][kw], kw = ceil(K/32): plane i holds
+ *                      bit i of every element (Section 3.1), element k of a row
+ *                      in word k/32 at bit k%32, pad bits zero.  This is the
+ *                      paper's depth-packed binary matrix (Algorithm 1) and, for
+ *                      activations, its channel-interleaved layout (Section 3.2).
+ *   QNN_FMT_INT8       one byte per element [rows][ld], ld = K rounded up to a
+ *                      multiple of 16, pad bytes zero: int8 for SIGNED/BIPOLAR,
+ *                      uint8 for UNSIGNED (Section 3: "casting all operands to
+ *                      8-bit integers"); the tensor-core path consumes this.
+ */
+#ifndef QNN_H_
+#define QNN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    QNN_OK = 0,
+    QNN_ERR_INVALID_ARG = -1,     /* null pointer, non-positive size, bad enum */
+    QNN_ERR_UNSUPPORTED = -2,     /* legal but not implemented combination    */
+    QNN_ERR_ALIGNMENT = -3,       /* a device pointer is not 16-byte aligned   */
+    QNN_ERR_WORKSPACE = -4,       /* workspace missing or too small            */
+    QNN_ERR_CUDA = -5,            /* a CUDA runtime/driver call failed         */
+    QNN_ERR_DEVICE_TIMEOUT = -6   /* a bounded device-side wait ran out        */
+} qnn_status;
+
+typedef enum { QNN_ENC_UNSIGNED = 0, QNN_ENC_SIGNED = 1, QNN_ENC_BIPOLAR = 2 } qnn_enc;
+typedef enum { QNN_FMT_BITPLANES = 0, QNN_FMT_INT8 = 1 } qnn_fmt;
+typedef enum { QNN_PATH_AUTO = 0, QNN_PATH_BITSERIAL = 1, QNN_PATH_TCGEN05_I8 = 2 } qnn_path;
+
+/* ---- packer (Section 3.1 bit planes; Section 3 8-bit containers) ---------- */
+
+typedef struct {
+    int rows;        /* M for weights, N for activations                      */
+    int K;           /* depth                                                 */
+    int bits;        /* 1..8; BIPOLAR requires 1                              */
+    int enc;         /* qnn_enc                                               */
+    int fmt;         /* qnn_fmt of the packed result                          */
+} qnn_pack_desc;
+
+/* Row pitch of a packed operand: 32-bit words per row and plane for BITPLANES
+ * (ceil(K/32)), bytes per row for INT8 (K rounded up to 16).  Host only. */
+size_t qnn_packed_ld(int K, int fmt);
+
+/* Bytes of a packed operand.  Host only; 0 on invalid arguments. */
+size_t qnn_packed_bytes(const qnn_pack_desc *d);
+
+/* logical: one byte per element, dense [rows][K] (uint8 for UNSIGNED, int8
+ * for SIGNED and BIPOLAR); values outside the encoding's range are truncated
+ * to their low `bits` bits (BIPOLAR: value > 0 -> bit 1).  packed: written in
+ * full, padding included.  Both 16-byte aligned. */
+qnn_status qnn_pack(const qnn_pack_desc *d, const void *logical, void *packed, void *stream);
+
+/* ---- fused GEMM + threshold (Sections 3.1 and 2.1.1) ---------------------- */
+
+typedef struct {
+    int M, N, K;
+    int w_bits, a_bits;   /* 1..8 (tensor path) / 1..4 (bit-serial path)      */
+    int out_bits;         /* 1..4: 2^out_bits - 1 thresholds per row; ignored
+                             when thr == NULL                                 */
+    int w_enc, a_enc;     /* qnn_enc                                          */
+    int w_fmt, a_fmt;     /* qnn_fmt; both operands must use the same format  */
+    int out_fmt;          /* qnn_fmt of the output codes; ignored if thr==NULL*/
+    int path;             /* qnn_path; AUTO selects by operand format         */
+} qnn_gemm_desc;
+
+/* Scratch bytes qnn_qgemm needs for this problem (may be 0).  Host only. */
+size_t qnn_gemm_workspace_bytes(const qnn_gemm_desc *d);
+
+/* Bytes of the output buffer for this problem (see qnn_qgemm).  Host only. */
+size_t qnn_gemm_out_bytes(const qnn_gemm_desc *d, int has_thresholds);
+
+/* acc[m][n] = sum_k W[m][k] * A[n][k], exact in int32 (Section 3.1), then
+ *   out[n][m] = #{ i : thr[m][i] <= acc[m][n] }      (Section 2.1.1, T(x, t)).
+ * thr: int32 [M][2^out_bits - 1], expected sorted non-decreasing per row (the
+ * counting rule is well defined either way).  Output, column(pixel)-major with
+ * channels fastest so that it is directly the next layer's activation operand:
+ *   out_fmt INT8       uint8  [N][ld], ld = M rounded up to 16, pad bytes 0
+ *   out_fmt BITPLANES  uint32 [out_bits][N][ceil(M/32)], pad bits 0
+ *   thr == NULL        int32  [N][M] raw accumulators
+ * The accumulators never reach global memory on the fused path.
+ * Errors: INVALID_ARG, UNSUPPORTED (mixed formats, bits out of range for the
+ * path, BIPOLAR with bits != 1), ALIGNMENT, WORKSPACE, CUDA. */
+qnn_status qnn_qgemm(const qnn_gemm_desc *d, const void *W, const void *A,
+                     const int32_t *thr, void *out,
+                     void *workspace, size_t workspace_bytes, void *stream);
+
+/* ---- lowering and convolution (Section 3.2) ------------------------------- */
+
+typedef struct {
+    int B, H, W, C;          /* input feature map, channels-last               */
+    int in_pitch;            /* INT8 only: bytes between consecutive pixels of
+                                the input map; 0 = C rounded up to 16          */
+    int OC, KH, KW;          /* filters                                        */
+    int stride, pad;         /* same in both spatial dimensions                */
+    int w_bits, a_bits, out_bits;
+    int w_enc, a_enc;
+    int fmt;                 /* qnn_fmt of input map, weights and lowered matrix */
+    int out_fmt;             /* qnn_fmt of the output map                      */
+    int path;                /* qnn_path                                       */
+} qnn_conv_desc;
+
+/* Output spatial size: (H + 2*pad - KH)/stride + 1.  Host only. */
+int qnn_conv_out_h(const qnn_conv_desc *d);
+int qnn_conv_out_w(const qnn_conv_desc *d);
+
+/* Depth of the lowered GEMM: BITPLANES -> 32 * KH*KW*ceil(C/32) (each pixel is
+ * padded to whole words, Section 3.2); INT8 -> KH*KW*C.  The weight operand
+ * passed to qnn_qconv must be packed with this K and the same per-pixel
+ * padding: logical weight row = (kh, kw, c) with c fastest.  Host only. */
+int qnn_conv_lowered_k(const qnn_conv_desc *d);
+
+/* Bytes of the lowered matrix / of qnn_qconv's workspace.  Host only. */
+size_t qnn_conv_lowered_bytes(const qnn_conv_desc *d);
+size_t qnn_conv_workspace_bytes(const qnn_conv_desc *d);
+size_t qnn_conv_out_bytes(const qnn_conv_desc *d, int has_thresholds);
+
+/* Interleaved lowering (Section 3.2): for every activation bit plane j and
+ * output pixel (b, oh, ow), concatenate over (kh, kw) in raster order the
+ * ceil(C/32) words of input pixel (oh*stride - pad + kh, ow*stride - pad + kw);
+ * pixels outside the image contribute zero words.
+ *   fmt BITPLANES: in uint32 [a_bits][B][H][W][ceil(C/32)]
+ *                  -> lowered uint32 [a_bits][B*OH*OW][KH*KW*ceil(C/32)]
+ *   fmt INT8:      in uint8 [B][H][W][in_pitch] (the first C bytes of a pixel
+ *                  are its channels) -> lowered uint8 [B*OH*OW][ld],
+ *                  ld = KH*KW*C rounded up to 16, pad bytes zero.
+ * The lowered matrix is the activation operand A of qnn_qgemm (N = B*OH*OW). */
+qnn_status qnn_im2col(const qnn_conv_desc *d, const void *in, void *lowered, void *stream);
+
+/* Convolution by lowering + fused GEMM/threshold.  Wpacked: the [OC][K_lowered]
+ * weight operand in format d->fmt.  Output: as qnn_qgemm with N = B*OH*OW,
+ * M = OC, i.e. a channels-last feature map [B][OH][OW][...].  BIPOLAR
+ * activations with pad > 0 are UNSUPPORTED (zero is not representable). */
+qnn_status qnn_qconv(const qnn_conv_desc *d, const void *Wpacked, const void *in,
+                     const int32_t *thr, void *out,
+                     void *workspace, size_t workspace_bytes, void *stream);
+
+/* ---- integer max-pool on activation codes (Section 4.2) ------------------- */
+
+typedef struct {
+    int B, H, W, C;      /* input map, channels-last                          */
+    int k, stride;       /* window and stride; no padding, floor              */
+    int bits;            /* code width (BITPLANES: number of planes)          */
+    int fmt;             /* INT8: uint8 [B][H][W][Cp], Cp = C rounded up to 16;
+                            BITPLANES: uint32 [bits][B][H][W][ceil(C/32)]     */
+} qnn_pool_desc;
+
+/* out has the same format with H, W replaced by (H-k)/stride+1, (W-k)/stride+1. */
+qnn_status qnn_maxpool(const qnn_pool_desc *d, const void *in, void *out, void *stream);
+
+/* ---- utilities ------------------------------------------------------------ */
+
+/* Checks on the device that every row of thr [M][n_thr] is sorted
+ * non-decreasing; *n_bad_rows receives the number of unsorted rows.
+ * SYNCHRONISES the stream. */
+qnn_status qnn_validate_thresholds(const int32_t *thr, int M, int n_thr,
+                                   int *n_bad_rows, void *stream);
+
+/* Reads and clears the device status word of the current device
+ * (QNN_OK or QNN_ERR_DEVICE_TIMEOUT).  SYNCHRONISES the device. */
+qnn_status qnn_device_status(int *status);
+
+/* Number of kernels this library has launched since it was loaded (host
+ * counter; used by benchmarks to report launches per step). */
+unsigned long long qnn_launch_count(void);
+
+const char *qnn_status_string(qnn_status s);
+int qnn_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QNN_H_ */

@@ -1,0 +1,45 @@
+// Shared host-side helpers of the qnn C ABI implementation (sm_100a only).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "qnn.h"
+
+namespace qnn {
+
+// Host counter of kernels launched by this library (reported by benchmarks).
+extern unsigned long long g_launches;
+
+inline void count_launch(int n = 1) { g_launches += (unsigned long long)n; }
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
+inline int ceil_div(int x, int m) { return (x + m - 1) / m; }
+
+inline bool valid_enc(int enc, int bits) {
+    if (enc == QNN_ENC_BIPOLAR) return bits == 1;
+    return enc == QNN_ENC_UNSIGNED || enc == QNN_ENC_SIGNED;
+}
+
+inline qnn_status launch_status() {
+    return cudaGetLastError() == cudaSuccess ? QNN_OK : QNN_ERR_CUDA;
+}
+
+// Number of SMs of the current device (cached per device).
+int sm_count();
+
+// Path implementations (one translation unit each).
+qnn_status pack_launch(const qnn_pack_desc *d, const void *logical, void *packed, cudaStream_t s);
+qnn_status gemm_bitserial_launch(const qnn_gemm_desc *d, const void *W, const void *A,
+                                 const int32_t *thr, void *out, cudaStream_t s);
+qnn_status gemm_tc_launch(const qnn_gemm_desc *d, const void *W, const void *A,
+                          const int32_t *thr, void *out, cudaStream_t s);
+qnn_status im2col_launch(const qnn_conv_desc *d, const void *in, void *lowered, cudaStream_t s);
+qnn_status maxpool_launch(const qnn_pool_desc *d, const void *in, void *out, cudaStream_t s);
+qnn_status validate_thresholds_launch(const int32_t *thr, int M, int n_thr, int *n_bad, cudaStream_t s);
+qnn_status device_status_read(int *status);
+
+}  // namespace qnn

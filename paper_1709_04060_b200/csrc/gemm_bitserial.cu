@@ -1,0 +1,225 @@
+// Bit-serial few-bit GEMM (Section 3.1, Algorithms 1 and 2) fused with the
+// threshold activation T(x, t) of Section 2.1.1.
+//
+// acc[m][n] = sum_i sum_j c_w[i] c_a[j] sum_d popc(W[i](m,d) & A[j](n,d)),
+// c[i] = +-2^i with the minus sign on the top plane of a SIGNED operand.
+// A BIPOLAR operand x = 2b - 1 is handled with b as its single plane:
+//   W bipolar:     acc = sum_j c_a[j] (2 popc(b & A[j]) - popc(A[j]))
+//   A bipolar:     acc = sum_i c_w[i] (2 popc(W[i] & b) - popc(W[i]))
+//   both bipolar:  acc = K - 2 popc(b_w ^ b_a)          (XNOR-popcount form)
+// The popc(A[j]) / popc(W[i]) correction sums are gathered while the tiles are
+// staged into shared memory, so they cost 1/64 of the main loop.
+//
+// Tiling: one CTA (8 warps) per 64 x 64 output tile, depth staged 16 words at a
+// time.  Lanes run along the output-channel dimension (rows m0+lane, m0+32+lane)
+// so that (a) weight words are read conflict-free from a 17-word-pitch tile while
+// activation words are warp-wide broadcasts, and (b) a warp ballot over the
+// bits of the 32 lanes' codes is exactly one word of the channel-interleaved
+// bit-plane layout of Section 3.2 that the next layer consumes.
+#include "common.cuh"
+
+namespace qnn {
+
+constexpr int BS_BM = 64, BS_BN = 64, BS_KT = 16, BS_PITCH = BS_KT + 1, BS_THREADS = 256;
+constexpr int BS_TN = 8;   // columns per warp
+
+struct BsParams {
+    const uint32_t *W;     // [WB][M][kw]
+    const uint32_t *A;     // [AB][N][kw]
+    const int32_t *thr;    // [M][n_thr] or null
+    void *out;
+    int M, N, K, kw;
+    int out_bits, out_fmt, ld_out;
+    int coef[4][4];        // multiplier of popc(W[i] op A[j])
+    int corr[4];           // multiplier of the correction popcounts (modes 1, 2)
+};
+
+enum { BS_REGULAR = 0, BS_W_BIPOLAR = 1, BS_A_BIPOLAR = 2, BS_BOTH_BIPOLAR = 3 };
+
+template <int WB, int AB, int MODE>
+__global__ void __launch_bounds__(BS_THREADS)
+qgemm_bitserial_kernel(const BsParams p) {
+    __shared__ uint32_t Ws[WB][BS_BM][BS_PITCH];
+    __shared__ uint32_t As[AB][BS_BN][BS_PITCH];
+    __shared__ int corr_s[64];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int m0 = blockIdx.y * BS_BM, n0 = blockIdx.x * BS_BN;
+    const int lc = tid & 15, lr = tid >> 4;      // staging: word column, first row
+
+    int acc[2][BS_TN];
+#pragma unroll
+    for (int t = 0; t < 2; ++t)
+#pragma unroll
+        for (int nn = 0; nn < BS_TN; ++nn) acc[t][nn] = 0;
+    int corr_part[4] = {0, 0, 0, 0};             // rows lr, lr+16, lr+32, lr+48
+
+    for (int kw0 = 0; kw0 < p.kw; kw0 += BS_KT) {
+        const int c = kw0 + lc;
+        const bool c_ok = c < p.kw;
+#pragma unroll
+        for (int i = 0; i < WB; ++i)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int r = lr + 16 * q, m = m0 + r;
+                uint32_t v = 0;
+                if (c_ok && m < p.M) v = p.W[((size_t)i * p.M + m) * p.kw + c];
+                Ws[i][r][lc] = v;
+                if (MODE == BS_A_BIPOLAR) corr_part[q] += p.corr[i] * __popc(v);
+            }
+#pragma unroll
+        for (int j = 0; j < AB; ++j)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int r = lr + 16 * q, n = n0 + r;
+                uint32_t v = 0;
+                if (c_ok && n < p.N) v = p.A[((size_t)j * p.N + n) * p.kw + c];
+                As[j][r][lc] = v;
+                if (MODE == BS_W_BIPOLAR) corr_part[q] += p.corr[j] * __popc(v);
+            }
+        __syncthreads();
+
+#pragma unroll 2
+        for (int cc = 0; cc < BS_KT; ++cc) {
+            uint32_t wv[2][WB];
+#pragma unroll
+            for (int t = 0; t < 2; ++t)
+#pragma unroll
+                for (int i = 0; i < WB; ++i) wv[t][i] = Ws[i][lane + 32 * t][cc];
+#pragma unroll
+            for (int nn = 0; nn < BS_TN; ++nn) {
+                uint32_t av[AB];
+#pragma unroll
+                for (int j = 0; j < AB; ++j) av[j] = As[j][warp * BS_TN + nn][cc];
+#pragma unroll
+                for (int t = 0; t < 2; ++t)
+#pragma unroll
+                    for (int i = 0; i < WB; ++i)
+#pragma unroll
+                        for (int j = 0; j < AB; ++j) {
+                            const uint32_t x = (MODE == BS_BOTH_BIPOLAR) ? (wv[t][i] ^ av[j])
+                                                                          : (wv[t][i] & av[j]);
+                            acc[t][nn] += p.coef[i][j] * __popc(x);
+                        }
+            }
+        }
+        __syncthreads();
+    }
+
+    // correction sums: reduce the 16 staging threads that share a row
+    if (MODE == BS_W_BIPOLAR || MODE == BS_A_BIPOLAR) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            int v = corr_part[q];
+#pragma unroll
+            for (int off = 8; off >= 1; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+            if (lc == 0) corr_s[lr + 16 * q] = v;
+        }
+        __syncthreads();
+    }
+
+    // epilogue: correction, threshold count, store
+    const int n_thr = p.thr ? (1 << p.out_bits) - 1 : 0;
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+        const int m = m0 + lane + 32 * t;
+        const bool m_ok = m < p.M;
+        int thr_r[15];
+#pragma unroll
+        for (int q = 0; q < 15; ++q)
+            thr_r[q] = (m_ok && q < n_thr) ? p.thr[(size_t)m * n_thr + q] : 0x7fffffff;
+#pragma unroll
+        for (int nn = 0; nn < BS_TN; ++nn) {
+            const int nl = warp * BS_TN + nn, n = n0 + nl;
+            int a = acc[t][nn];
+            if (MODE == BS_W_BIPOLAR) a -= corr_s[nl];
+            if (MODE == BS_A_BIPOLAR) a -= corr_s[lane + 32 * t];
+            if (MODE == BS_BOTH_BIPOLAR) a += p.K;
+            if (n >= p.N) continue;                       // warp-uniform
+            if (!p.thr) {
+                if (m_ok) reinterpret_cast<int32_t *>(p.out)[(size_t)n * p.M + m] = a;
+                continue;
+            }
+            int code = 0;
+#pragma unroll
+            for (int q = 0; q < 15; ++q) code += (a >= thr_r[q]) ? 1 : 0;   // pads are INT32_MAX
+            if (!m_ok) code = 0;
+            if (p.out_fmt == QNN_FMT_INT8) {
+                if (m < p.ld_out) reinterpret_cast<uint8_t *>(p.out)[(size_t)n * p.ld_out + m] = (uint8_t)code;
+            } else {
+                const int mw = (p.M + 31) >> 5, word = (m0 >> 5) + t;
+                for (int b = 0; b < p.out_bits; ++b) {
+                    const uint32_t bits = __ballot_sync(0xffffffffu, (code >> b) & 1);
+                    if (lane == 0 && word < mw)
+                        reinterpret_cast<uint32_t *>(p.out)[((size_t)b * p.N + n) * mw + word] = bits;
+                }
+            }
+        }
+    }
+}
+
+template <int WB, int AB, int MODE>
+static void launch_one(const BsParams &p, cudaStream_t s) {
+    dim3 grid(ceil_div(p.N, BS_BN), ceil_div(p.M, BS_BM));
+    qgemm_bitserial_kernel<WB, AB, MODE><<<grid, BS_THREADS, 0, s>>>(p);
+}
+
+template <int MODE>
+static bool dispatch_bits(int wb, int ab, const BsParams &p, cudaStream_t s) {
+#define QNN_BS_CASE(W_, A_) if (wb == W_ && ab == A_) { launch_one<W_, A_, MODE>(p, s); return true; }
+    if (MODE == BS_REGULAR) {
+        QNN_BS_CASE(1, 1) QNN_BS_CASE(1, 2) QNN_BS_CASE(1, 3) QNN_BS_CASE(1, 4)
+        QNN_BS_CASE(2, 1) QNN_BS_CASE(2, 2) QNN_BS_CASE(2, 3) QNN_BS_CASE(2, 4)
+        QNN_BS_CASE(3, 1) QNN_BS_CASE(3, 2) QNN_BS_CASE(3, 3) QNN_BS_CASE(3, 4)
+        QNN_BS_CASE(4, 1) QNN_BS_CASE(4, 2) QNN_BS_CASE(4, 3) QNN_BS_CASE(4, 4)
+    } else if (MODE == BS_W_BIPOLAR) {
+        QNN_BS_CASE(1, 1) QNN_BS_CASE(1, 2) QNN_BS_CASE(1, 3) QNN_BS_CASE(1, 4)
+    } else if (MODE == BS_A_BIPOLAR) {
+        QNN_BS_CASE(1, 1) QNN_BS_CASE(2, 1) QNN_BS_CASE(3, 1) QNN_BS_CASE(4, 1)
+    } else {
+        QNN_BS_CASE(1, 1)
+    }
+#undef QNN_BS_CASE
+    return false;
+}
+
+// Plane weights: +2^i, minus on the top plane of a SIGNED operand (Algorithm 2).
+static void plane_coef(int bits, int enc, int *c) {
+    for (int i = 0; i < 4; ++i) c[i] = 0;
+    for (int i = 0; i < bits; ++i) c[i] = (enc == QNN_ENC_SIGNED && i == bits - 1) ? -(1 << i) : (1 << i);
+}
+
+qnn_status gemm_bitserial_launch(const qnn_gemm_desc *d, const void *W, const void *A,
+                                 const int32_t *thr, void *out, cudaStream_t s) {
+    BsParams p;
+    p.W = (const uint32_t *)W; p.A = (const uint32_t *)A; p.thr = thr; p.out = out;
+    p.M = d->M; p.N = d->N; p.K = d->K; p.kw = ceil_div(d->K, 32);
+    p.out_bits = thr ? d->out_bits : 0;
+    p.out_fmt = d->out_fmt;
+    p.ld_out = round_up(d->M, 16);
+    int cw[4], ca[4];
+    plane_coef(d->w_bits, d->w_enc, cw);
+    plane_coef(d->a_bits, d->a_enc, ca);
+    const bool wb = d->w_enc == QNN_ENC_BIPOLAR, ab = d->a_enc == QNN_ENC_BIPOLAR;
+    for (int i = 0; i < 4; ++i) p.corr[i] = 0;
+    for (int i = 0; i < 4; ++i)
+        for (int j = 0; j < 4; ++j) p.coef[i][j] = cw[i] * ca[j];
+    bool ok;
+    if (wb && ab) {
+        p.coef[0][0] = -2;
+        ok = dispatch_bits<BS_BOTH_BIPOLAR>(1, 1, p, s);
+    } else if (wb) {
+        for (int j = 0; j < 4; ++j) { p.coef[0][j] = 2 * ca[j]; p.corr[j] = ca[j]; }
+        ok = dispatch_bits<BS_W_BIPOLAR>(1, d->a_bits, p, s);
+    } else if (ab) {
+        for (int i = 0; i < 4; ++i) { p.coef[i][0] = 2 * cw[i]; p.corr[i] = cw[i]; }
+        ok = dispatch_bits<BS_A_BIPOLAR>(d->w_bits, 1, p, s);
+    } else {
+        ok = dispatch_bits<BS_REGULAR>(d->w_bits, d->a_bits, p, s);
+    }
+    if (!ok) return QNN_ERR_UNSUPPORTED;
+    count_launch();
+    return launch_status();
+}
+
+}  // namespace qnn

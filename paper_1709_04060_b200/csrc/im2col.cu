@@ -1,0 +1,158 @@
+// Interleaved lowering (Section 3.2): the feature map is channels-last, one
+// bit position per plane, every pixel padded to whole words, so lowering moves
+// whole words -- one im2col per activation bit plane, no masking or shifting.
+// The same kernel lowers 8-bit-container maps in 16-byte units (channel count a
+// multiple of 16); a byte-granular variant covers other channel counts (the
+// 3-channel input image of the first layer).
+//
+// One warp per output pixel: the pixel's coordinates are decoded once, lanes
+// stream the lowered row (kh, kw, c order, c fastest) with coalesced stores.
+#include "common.cuh"
+
+namespace qnn {
+
+struct FastDiv {          // exact n / d for n, d < 65536
+    uint32_t d, magic;
+};
+static FastDiv make_fastdiv(int d) {
+    FastDiv f;
+    f.d = (uint32_t)d;
+    f.magic = (uint32_t)(((1ull << 32) + (uint64_t)d - 1) / (uint64_t)d);
+    return f;
+}
+__device__ __forceinline__ uint32_t fdiv(uint32_t n, FastDiv f) {
+    return f.d == 1 ? n : __umulhi(n, f.magic);
+}
+
+struct LowerParams {
+    const void *in;
+    void *out;
+    int planes;                 // bit planes (1 for 8-bit containers)
+    int B, H, W, OH, OW;
+    int KH, KW, stride, pad;
+    int cu;                     // units per pixel that are copied
+    int pitch;                  // units between consecutive input pixels
+    int row_units;              // units per lowered row that are written
+    int row_copy;               // KH*KW*cu: units per lowered row that carry data
+    long long npix;             // B*OH*OW
+    FastDiv seg, cud, ohow, owd;
+};
+
+template <typename T>
+__device__ __forceinline__ T zero_unit();
+template <> __device__ __forceinline__ uint32_t zero_unit<uint32_t>() { return 0u; }
+template <> __device__ __forceinline__ uint4 zero_unit<uint4>() { return make_uint4(0, 0, 0, 0); }
+
+template <typename T>
+__global__ void __launch_bounds__(256) lower_units_kernel(const LowerParams p) {
+    const int lane = threadIdx.x & 31;
+    const long long warp0 = (blockIdx.x * (long long)blockDim.x + threadIdx.x) >> 5;
+    const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+    const T *in = reinterpret_cast<const T *>(p.in);
+    T *out = reinterpret_cast<T *>(p.out);
+    const long long total = p.npix * p.planes;
+    for (long long job = warp0; job < total; job += nwarps) {
+        const int plane = (int)(job / p.npix);
+        const long long pix = job - (long long)plane * p.npix;
+        const int b = (int)(pix / (p.OH * p.OW));
+        const uint32_t rem = (uint32_t)(pix - (long long)b * p.OH * p.OW);
+        const int oh = (int)fdiv(rem, p.owd), ow = (int)(rem - oh * p.OW);
+        const int ih0 = oh * p.stride - p.pad, iw0 = ow * p.stride - p.pad;
+        const T *src = in + ((size_t)plane * p.B + b) * p.H * p.W * p.pitch;
+        T *dst = out + (size_t)job * p.row_units;
+        for (int w = lane; w < p.row_units; w += 32) {
+            T v = zero_unit<T>();
+            if (w < p.row_copy) {
+                const int kh = (int)fdiv(w, p.seg), r = w - kh * (int)p.seg.d;
+                const int kw = (int)fdiv(r, p.cud), c = r - kw * p.cu;
+                const int ih = ih0 + kh, iw = iw0 + kw;
+                if (ih >= 0 && ih < p.H && iw >= 0 && iw < p.W)
+                    v = src[((size_t)ih * p.W + iw) * p.pitch + c];
+            }
+            dst[w] = v;
+        }
+    }
+}
+
+// Byte-granular lowering of 8-bit maps: a thread assembles 4 consecutive output bytes.
+__global__ void __launch_bounds__(256) lower_bytes_kernel(const LowerParams p) {
+    const int lane = threadIdx.x & 31;
+    const long long warp0 = (blockIdx.x * (long long)blockDim.x + threadIdx.x) >> 5;
+    const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+    const uint8_t *in = reinterpret_cast<const uint8_t *>(p.in);
+    uint32_t *out = reinterpret_cast<uint32_t *>(p.out);
+    const int row_words = p.row_units >> 2;        // row pitch is a multiple of 16 bytes
+    for (long long pix = warp0; pix < p.npix; pix += nwarps) {
+        const int b = (int)(pix / (p.OH * p.OW));
+        const uint32_t rem = (uint32_t)(pix - (long long)b * p.OH * p.OW);
+        const int oh = (int)fdiv(rem, p.owd), ow = (int)(rem - oh * p.OW);
+        const int ih0 = oh * p.stride - p.pad, iw0 = ow * p.stride - p.pad;
+        const uint8_t *src = in + (size_t)b * p.H * p.W * p.pitch;
+        uint32_t *dst = out + (size_t)pix * row_words;
+        for (int q = lane; q < row_words; q += 32) {
+            int k = q * 4;
+            int kh = (int)fdiv(k, p.seg), r = k - kh * (int)p.seg.d;
+            int kw = (int)fdiv(r, p.cud), c = r - kw * p.cu;
+            uint32_t v = 0;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                if (k + e < p.row_copy) {
+                    const int ih = ih0 + kh, iw = iw0 + kw;
+                    if (ih >= 0 && ih < p.H && iw >= 0 && iw < p.W)
+                        v |= (uint32_t)src[((size_t)ih * p.W + iw) * p.pitch + c] << (8 * e);
+                }
+                if (++c == p.cu) { c = 0; if (++kw == p.KW) { kw = 0; ++kh; } }
+            }
+            dst[q] = v;
+        }
+    }
+}
+
+qnn_status im2col_launch(const qnn_conv_desc *d, const void *in, void *lowered, cudaStream_t s) {
+    LowerParams p;
+    p.in = in; p.out = lowered;
+    p.B = d->B; p.H = d->H; p.W = d->W;
+    p.OH = qnn_conv_out_h(d); p.OW = qnn_conv_out_w(d);
+    p.KH = d->KH; p.KW = d->KW; p.stride = d->stride; p.pad = d->pad;
+    p.npix = (long long)d->B * p.OH * p.OW;
+    if (p.OH * p.OW >= 65536 || p.OW >= 65536) return QNN_ERR_UNSUPPORTED;
+    p.owd = make_fastdiv(p.OW);
+    p.ohow = make_fastdiv(1);
+    const int threads = 256;
+    const long long max_blocks = (long long)sm_count() * 16;
+
+    int mode;   // 0 words, 1 16-byte units, 2 bytes
+    if (d->fmt == QNN_FMT_BITPLANES) {
+        mode = 0;
+        p.planes = d->a_bits;
+        p.cu = ceil_div(d->C, 32); p.pitch = p.cu;
+        p.row_copy = d->KH * d->KW * p.cu; p.row_units = p.row_copy;
+    } else {
+        const int pitch = d->in_pitch ? d->in_pitch : round_up(d->C, 16);
+        const int ld = round_up(d->KH * d->KW * d->C, 16);
+        p.planes = 1;
+        if (d->C % 16 == 0 && pitch % 16 == 0) {
+            mode = 1;
+            p.cu = d->C / 16; p.pitch = pitch / 16;
+            p.row_copy = d->KH * d->KW * p.cu; p.row_units = ld / 16;
+        } else {
+            mode = 2;
+            p.cu = d->C; p.pitch = pitch;
+            p.row_copy = d->KH * d->KW * d->C; p.row_units = ld;
+        }
+    }
+    if (p.row_units >= 65536 || d->KW * p.cu >= 65536) return QNN_ERR_UNSUPPORTED;
+    p.seg = make_fastdiv(d->KW * p.cu);
+    p.cud = make_fastdiv(p.cu);
+
+    const long long jobs = p.npix * p.planes;
+    long long blocks = (jobs * 32 + threads - 1) / threads;
+    if (blocks > max_blocks) blocks = max_blocks;
+    if (mode == 0) lower_units_kernel<uint32_t><<<(unsigned)blocks, threads, 0, s>>>(p);
+    else if (mode == 1) lower_units_kernel<uint4><<<(unsigned)blocks, threads, 0, s>>>(p);
+    else lower_bytes_kernel<<<(unsigned)blocks, threads, 0, s>>>(p);
+    count_launch();
+    return launch_status();
+}
+
+}  // namespace qnn

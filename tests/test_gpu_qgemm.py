@@ -1,0 +1,136 @@
+"""GPU parity: packer and fused GEMM+threshold through the C ABI vs the CPU oracle.
+Bit-exact on every element (integer results are unique)."""
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as orc
+from paper_1709_04060_b200 import synth
+from qnn_testutil import unpack_operand, decode_out
+
+pytestmark = pytest.mark.gpu
+
+BITPLANES, INT8 = 0, 1
+
+
+@pytest.fixture(scope="module")
+def qb():
+    from paper_1709_04060_b200 import binding
+    return binding
+
+
+def run_case(qb, case, fmt, out_fmt, raw=False, path=0, check_pack=False):
+    Wd = qb.to_device_logical(case.W, case.w_enc)
+    Ad = qb.to_device_logical(case.At, case.a_enc)
+    Wp = qb.pack(Wd, case.w_bits, case.w_enc, fmt)
+    Ap = qb.pack(Ad, case.a_bits, case.a_enc, fmt)
+    if check_pack:
+        w_back = unpack_operand(Wp.cpu().numpy(), fmt, case.w_bits, case.M, case.K, case.w_enc)
+        a_back = unpack_operand(Ap.cpu().numpy(), fmt, case.a_bits, case.N, case.K, case.a_enc)
+        assert np.array_equal(w_back, case.W) and np.array_equal(a_back, case.At)
+    thr = None if raw else torch.from_numpy(case.thr).cuda()
+    d = qb.gemm_desc(case.M, case.N, case.K, case.w_bits, case.a_bits, case.out_bits,
+                     case.w_enc, case.a_enc, fmt, out_fmt, path)
+    out = qb.qgemm(d, Wp, Ap, thr)
+    torch.cuda.synchronize()
+    st, dev = qb.qnn_device_status()
+    assert st == 0 and dev == 0
+    got = decode_out(out.cpu().numpy().view(np.uint8).reshape(-1), out_fmt, case.out_bits,
+                     case.N, case.M, raw)
+    want = orc.qgemm(case.W, case.At, None if raw else case.thr).T
+    assert got.shape == want.shape
+    bad = np.argwhere(got != want)
+    assert bad.size == 0, f"{len(bad)} mismatches, first at (n,m)={bad[0]}: got {got[tuple(bad[0])]} want {want[tuple(bad[0])]}"
+
+
+@pytest.mark.parametrize("fmt", [BITPLANES, INT8])
+@pytest.mark.parametrize("out_fmt,raw", [(INT8, False), (BITPLANES, False), (INT8, True)])
+def test_config1_w1a2(qb, fmt, out_fmt, raw):
+    """Single W1A2 GEMM+threshold: M=64, K=576 bipolar weights, N=256 2-bit activations."""
+    case = synth.gemm_case(1, 64, 256, 576, 1, 2)
+    run_case(qb, case, fmt, out_fmt, raw, check_pack=True)
+
+
+@pytest.mark.parametrize("fmt", [BITPLANES, INT8])
+def test_config1_full_range_thresholds_with_ties(qb, fmt):
+    """Thresholds over the whole +-1728 accumulator range, duplicates, and values
+    that accumulators hit exactly (ties count as passed)."""
+    case = synth.gemm_case(1, 64, 256, 576, 1, 2, spread=38.5)
+    acc = orc.gemm(case.W, case.At)
+    thr = case.thr.copy()
+    thr[0] = [acc[0, 0], acc[0, 0], acc[0, 1]]
+    thr[0].sort()
+    thr[1] = [-1728, 0, 1728]
+    thr[2] = [-(2**31), -(2**31), 2**31 - 1]
+    thr[3] = [int(acc[3].min()), int(np.median(acc[3])), int(acc[3].max())]
+    case.thr = thr
+    run_case(qb, case, fmt, INT8)
+    run_case(qb, case, fmt, BITPLANES)
+
+
+@pytest.mark.parametrize("fmt", [BITPLANES, INT8])
+@pytest.mark.parametrize("w_bits,a_bits", list(itertools.product((1, 2, 3, 4), repeat=2)))
+def test_all_widths_ragged(qb, fmt, w_bits, a_bits):
+    """Every (w, a) pair with each encoding, on sizes that span several tiles of
+    both kernels and leave ragged tails in M, N and K."""
+    w_encs = [synth.SIGNED, synth.UNSIGNED] + ([synth.BIPOLAR] if w_bits == 1 else [])
+    a_encs = [synth.UNSIGNED, synth.SIGNED] + ([synth.BIPOLAR] if a_bits == 1 else [])
+    seed = 200 + 10 * w_bits + a_bits
+    for w_enc, a_enc in itertools.product(w_encs, a_encs):
+        case = synth.gemm_case(seed, 197, 301, 1100, w_bits, a_bits, w_enc, a_enc, out_bits=a_bits)
+        out_fmt = BITPLANES if (w_enc + a_enc) % 2 else INT8
+        run_case(qb, case, fmt, out_fmt, check_pack=True)
+
+
+@pytest.mark.parametrize("fmt", [BITPLANES, INT8])
+@pytest.mark.parametrize("M,N,K", [(1, 1, 1), (1, 7, 33), (129, 1, 31), (130, 257, 129),
+                                   (64, 513, 4100), (300, 40, 16)])
+def test_edge_shapes(qb, fmt, M, N, K):
+    case = synth.gemm_case(300 + M + N, M, N, K, 2, 2)
+    run_case(qb, case, fmt, INT8, check_pack=True)
+    run_case(qb, case, fmt, BITPLANES)
+    run_case(qb, case, fmt, INT8, raw=True)
+
+
+@pytest.mark.parametrize("out_bits", [1, 2, 3, 4])
+def test_out_bits_independent_of_a_bits(qb, out_bits):
+    for fmt in (BITPLANES, INT8):
+        case = synth.gemm_case(400 + out_bits, 150, 200, 640, 2, 3, out_bits=out_bits)
+        run_case(qb, case, fmt, INT8)
+        run_case(qb, case, fmt, BITPLANES)
+
+
+def test_eight_bit_layers_tensor_path(qb):
+    """8-bit first/last layer shapes (Section 4.2): s8 x u8 with K=363 (not a
+    multiple of 16) and thresholds; s8 x 2-bit codes with raw int32 output."""
+    c1 = synth.gemm_case(500, 96, 3025, 363, 8, 8, synth.SIGNED, synth.UNSIGNED, out_bits=2)
+    run_case(qb, c1, INT8, INT8, check_pack=True)
+    c8 = synth.gemm_case(501, 1000, 5, 4096, 8, 2, synth.SIGNED, synth.UNSIGNED, out_bits=2)
+    run_case(qb, c8, INT8, INT8, raw=True)
+
+
+def test_unsorted_thresholds_follow_counting_rule(qb):
+    case = synth.gemm_case(600, 70, 90, 256, 2, 2)
+    case.thr = case.thr[:, ::-1].copy()
+    for fmt in (BITPLANES, INT8):
+        run_case(qb, case, fmt, INT8)
+    st, bad = qb.qnn_validate_thresholds(torch.from_numpy(case.thr).cuda(), 70, 3)
+    assert st == 0 and bad == int((np.diff(case.thr, axis=1) < 0).any(axis=1).sum())
+    st, bad = qb.qnn_validate_thresholds(torch.from_numpy(np.sort(case.thr, axis=1)).cuda(), 70, 3)
+    assert st == 0 and bad == 0
+
+
+def test_outputs_monotone_in_accumulator(qb):
+    """Codes are non-decreasing in the raw accumulator (property, any size)."""
+    case = synth.gemm_case(700, 256, 512, 2048, 1, 2)
+    Wd = qb.to_device_logical(case.W, case.w_enc)
+    Ad = qb.to_device_logical(case.At, case.a_enc)
+    Wp, Ap = qb.pack(Wd, 1, case.w_enc, INT8), qb.pack(Ad, 2, case.a_enc, INT8)
+    d = qb.gemm_desc(256, 512, 2048, 1, 2, 2, case.w_enc, case.a_enc, INT8, INT8)
+    codes = qb.qgemm(d, Wp, Ap, torch.from_numpy(case.thr).cuda()).cpu().numpy()[: 512 * 256].reshape(512, 256)
+    acc = qb.qgemm(d, Wp, Ap, None).cpu().numpy()
+    for m in range(0, 256, 17):
+        order = np.argsort(acc[:, m], kind="stable")
+        assert np.all(np.diff(codes[order, m].astype(np.int32)) >= 0)
