@@ -62,6 +62,11 @@ static qnn_status check_conv_desc(const qnn_conv_desc *d) {
     if (d->H + 2 * d->pad < d->KH || d->W + 2 * d->pad < d->KW) return QNN_ERR_INVALID_ARG;
     if (d->fmt == QNN_FMT_INT8 && d->in_pitch != 0 && d->in_pitch < d->C) return QNN_ERR_INVALID_ARG;
     if (d->a_enc == QNN_ENC_BIPOLAR && d->pad > 0) return QNN_ERR_UNSUPPORTED;
+    // per-pixel pad bits would read as -1 for a bipolar operand
+    if (d->fmt == QNN_FMT_BITPLANES && (d->C % 32) != 0 &&
+        (d->a_enc == QNN_ENC_BIPOLAR || d->w_enc == QNN_ENC_BIPOLAR) &&
+        (d->a_enc == QNN_ENC_BIPOLAR) == (d->w_enc == QNN_ENC_BIPOLAR))
+        return QNN_ERR_UNSUPPORTED;
     return QNN_OK;
 }
 

@@ -1,0 +1,194 @@
+"""GPU parity: interleaved lowering, convolution by lowering, max-pool and the
+AlexNet-shaped chain through the C ABI vs the CPU oracle (bit-exact)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as orc
+from oracle import alexnet as onet
+from paper_1709_04060_b200 import synth
+from qnn_testutil import unpack_planes, unpack_int8, decode_out, round_up
+
+pytestmark = pytest.mark.gpu
+
+BITPLANES, INT8 = 0, 1
+
+
+@pytest.fixture(scope="module")
+def qb():
+    from paper_1709_04060_b200 import binding
+    return binding
+
+
+def host_im2col(In, KH, KW, stride, pad, c_pad):
+    """Test-side lowering: rows (b, oh, ow), columns (kh, kw, c) with each pixel padded to c_pad."""
+    B, H, Wd, C = In.shape
+    OH = (H + 2 * pad - KH) // stride + 1
+    OW = (Wd + 2 * pad - KW) // stride + 1
+    padded = np.zeros((B, H + 2 * pad, Wd + 2 * pad, c_pad), dtype=In.dtype)
+    padded[:, pad:pad + H, pad:pad + Wd, :C] = In
+    cols = np.empty((B, OH, OW, KH, KW, c_pad), dtype=In.dtype)
+    for oh in range(OH):
+        for ow in range(OW):
+            cols[:, oh, ow] = padded[:, oh * stride:oh * stride + KH, ow * stride:ow * stride + KW, :]
+    return cols.reshape(B * OH * OW, KH * KW * c_pad)
+
+
+def device_map(qb, case, fmt, in_pitch=None):
+    """Feature map on the device in the library's layout; returns (tensor, pitch)."""
+    B, H, Wd, C = case.In.shape
+    if fmt == BITPLANES:
+        flat = qb.to_device_logical(case.In.reshape(B * H * Wd, C), case.a_enc)
+        return qb.pack(flat, case.a_bits, case.a_enc, BITPLANES), 0
+    pitch = in_pitch if in_pitch is not None else round_up(C, 16)
+    m = np.zeros((B, H, Wd, pitch), dtype=np.uint8)
+    m[..., :C] = case.In.astype(np.uint8)
+    return torch.from_numpy(m).cuda(), pitch
+
+
+def device_weights(qb, case, fmt):
+    OC, KH, KW, C = case.Wt.shape
+    if fmt == BITPLANES:
+        cp = round_up(C, 32)
+        Wp = np.zeros((OC, KH * KW, cp), dtype=np.int32)
+        Wp[:, :, :C] = case.Wt.reshape(OC, KH * KW, C)
+        flat = Wp.reshape(OC, -1)
+    else:
+        flat = case.Wt.reshape(OC, -1)
+    return qb.pack(qb.to_device_logical(flat, case.w_enc), case.w_bits, case.w_enc, fmt)
+
+
+def conv_desc(qb, case, fmt, out_fmt, pitch):
+    return qb.qnn_conv_desc(case.B, case.H, case.Wd, case.C, pitch, case.OC, case.KH, case.KW,
+                            case.stride, case.pad, case.w_bits, case.a_bits, case.out_bits,
+                            case.w_enc, case.a_enc, fmt, out_fmt, 0)
+
+
+CONV_CASES = [
+    # B, H, W, C, OC, KH, KW, stride, pad, w_bits, a_bits
+    (2, 9, 9, 96, 70, 5, 5, 1, 2, 1, 2),
+    (1, 13, 11, 40, 33, 3, 3, 1, 1, 2, 2),      # C not a multiple of 32 / 16
+    (3, 12, 12, 32, 64, 3, 3, 2, 0, 1, 2),
+    (1, 8, 8, 256, 130, 1, 1, 1, 0, 4, 4),
+    (2, 7, 7, 64, 16, 7, 7, 1, 3, 3, 1),
+]
+
+
+@pytest.mark.parametrize("fmt", [BITPLANES, INT8])
+@pytest.mark.parametrize("shape", CONV_CASES)
+def test_im2col_matches_host_lowering(qb, fmt, shape):
+    case = synth.conv_case(800 + shape[3], *shape)
+    x, pitch = device_map(qb, case, fmt)
+    d = conv_desc(qb, case, fmt, INT8, pitch)
+    npix = case.B * case.OH * case.OW
+    low = torch.full((qb.qnn_conv_lowered_bytes(d),), 0xAB, dtype=torch.uint8, device="cuda")
+    qb.check(qb.qnn_im2col(d, x, low))
+    torch.cuda.synchronize()
+    K = qb.qnn_conv_lowered_k(d)
+    if fmt == BITPLANES:
+        got = unpack_planes(low.cpu().numpy(), case.a_bits, npix, K, case.a_enc)
+        want = host_im2col(case.In, case.KH, case.KW, case.stride, case.pad, round_up(case.C, 32))
+    else:
+        got = unpack_int8(low.cpu().numpy(), npix, K, case.a_enc)
+        want = host_im2col(case.In, case.KH, case.KW, case.stride, case.pad, case.C)
+    assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("fmt", [BITPLANES, INT8])
+@pytest.mark.parametrize("out_fmt", [BITPLANES, INT8])
+@pytest.mark.parametrize("shape", CONV_CASES)
+def test_qconv_matches_direct_convolution(qb, fmt, out_fmt, shape):
+    case = synth.conv_case(900 + shape[4], *shape)
+    x, pitch = device_map(qb, case, fmt)
+    Wp = device_weights(qb, case, fmt)
+    d = conv_desc(qb, case, fmt, out_fmt, pitch)
+    out = qb.qconv(d, Wp, x, torch.from_numpy(case.thr).cuda())
+    torch.cuda.synchronize()
+    npix = case.B * case.OH * case.OW
+    got = decode_out(out.cpu().numpy(), out_fmt, case.out_bits, npix, case.OC, False)
+    want = orc.qconv(case.In, case.Wt, case.thr, case.stride, case.pad).reshape(npix, case.OC)
+    assert np.array_equal(got, want)
+    raw = qb.qconv(d, Wp, x, None)
+    torch.cuda.synchronize()
+    got = decode_out(raw.cpu().numpy(), out_fmt, case.out_bits, npix, case.OC, True)
+    assert np.array_equal(got, orc.conv_direct(case.In, case.Wt, case.stride, case.pad).reshape(npix, case.OC))
+
+
+@pytest.mark.parametrize("fmt", [BITPLANES, INT8])
+@pytest.mark.parametrize("B", [1, 4])
+def test_config3_conv2_alexnet_shape(qb, fmt, B):
+    """AlexNet conv2-shaped W1A2 layer: lowered GEMM rows 256, depth 2400, cols 729 per image."""
+    case = synth.conv2_alexnet_case(B)
+    x, pitch = device_map(qb, case, fmt)
+    Wp = device_weights(qb, case, fmt)
+    d = conv_desc(qb, case, fmt, INT8, pitch)
+    assert qb.qnn_conv_lowered_k(d) == 2400
+    out = qb.qconv(d, Wp, x, torch.from_numpy(case.thr).cuda())
+    torch.cuda.synchronize()
+    got = decode_out(out.cpu().numpy(), INT8, 2, B * 729, 256, False)
+    want = orc.qconv(case.In, case.Wt, case.thr, 1, 2).reshape(B * 729, 256)
+    assert np.array_equal(got, want)
+    assert len(np.unique(got)) == 4
+
+
+def test_conv1_shape_byte_lowering(qb):
+    """First-layer shape: 3-channel uint8 image with pixel pitch 3, 11x11 stride 4 (K=363)."""
+    case = synth.conv_case(950, 2, 227, 227, 3, 96, 11, 11, 4, 0, 8, 8, synth.SIGNED, synth.UNSIGNED)
+    x, pitch = device_map(qb, case, INT8, in_pitch=3)
+    Wp = device_weights(qb, case, INT8)
+    for out_fmt in (INT8, BITPLANES):
+        d = conv_desc(qb, case, INT8, out_fmt, pitch)
+        out = qb.qconv(d, Wp, x, torch.from_numpy(case.thr).cuda())
+        torch.cuda.synchronize()
+        got = decode_out(out.cpu().numpy(), out_fmt, 2, 2 * 3025, 96, False)
+        want = orc.qconv(case.In, case.Wt, case.thr, 4, 0).reshape(2 * 3025, 96)
+        assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("fmt", [BITPLANES, INT8])
+@pytest.mark.parametrize("B,H,C,bits", [(2, 55, 96, 2), (1, 13, 256, 2), (3, 9, 40, 4), (1, 7, 33, 3), (2, 5, 64, 1)])
+def test_maxpool(qb, fmt, B, H, C, bits):
+    rng = np.random.default_rng(B * 100 + H)
+    codes = rng.integers(0, 1 << bits, size=(B, H, H, C), dtype=np.int32)
+    OH = (H - 3) // 2 + 1
+    want = orc.maxpool(codes, 3, 2)
+    if fmt == BITPLANES:
+        x = qb.pack(qb.to_device_logical(codes.reshape(-1, C), 0), bits, 0, BITPLANES)
+        out = torch.empty(bits * B * OH * OH * ((C + 31) // 32) * 4, dtype=torch.uint8, device="cuda")
+    else:
+        cp = round_up(C, 16)
+        m = np.zeros((B, H, H, cp), dtype=np.uint8)
+        m[..., :C] = codes
+        x = torch.from_numpy(m).cuda()
+        out = torch.empty(B * OH * OH * cp, dtype=torch.uint8, device="cuda")
+    d = qb.qnn_pool_desc(B, H, H, C, 3, 2, bits, fmt)
+    qb.check(qb.qnn_maxpool(d, x, out))
+    torch.cuda.synchronize()
+    got = decode_out(out.cpu().numpy(), fmt, bits, B * OH * OH, C, False)
+    assert np.array_equal(got, want.reshape(-1, C))
+
+
+@pytest.mark.parametrize("mode", ["tensor", "bitserial"])
+@pytest.mark.parametrize("B", [1, 3])
+def test_alexnet_chain_per_layer(qb, mode, B):
+    """Every intermediate activation tensor and the final logits vs the oracle chain."""
+    from paper_1709_04060_b200.alexnet import AlexNetPlan
+    net = synth.alexnet_case(B)
+    logits_ref, inter_ref = onet.forward(net)
+    plan = AlexNetPlan(net, B, mode)
+    img = torch.from_numpy(net.image.astype(np.uint8)).cuda()
+    logits = plan.forward(img)
+    torch.cuda.synchronize()
+    st, dev = qb.qnn_device_status()
+    assert st == 0 and dev == 0
+    inter = plan.intermediates()
+    for L in net.layers[:-1]:
+        name = L.name + "_pool" if L.pool else L.name
+        buf, kind, d = inter[name]
+        want = inter_ref[L.name]
+        C = want.shape[-1]
+        npix = want.size // C
+        fmt = d.fmt if kind == "pool" else d.out_fmt
+        got = decode_out(buf.cpu().numpy(), fmt, 2, npix, C, False)
+        assert np.array_equal(got, want.reshape(npix, C)), f"{mode}: first mismatch after {L.name}"
+    assert np.array_equal(logits.cpu().numpy().astype(np.int64), logits_ref)
