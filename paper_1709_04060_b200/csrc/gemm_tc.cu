@@ -21,6 +21,7 @@
 // main loop of tile t+1.  Every wait is bounded; on expiry the CTA records
 // QNN_ERR_DEVICE_TIMEOUT in the device status word, drains and exits.
 #include <cuda.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 
@@ -129,11 +130,101 @@ struct TcParams {
     int M, N, K;
     int tiles_m, tiles_n, num_kb;
     int ld_out;            // INT8 output row pitch
+    int fp_count;          // 1: |acc| < 2^24, thresholds are counted on the FP32 pipe
     uint32_t idesc;
 };
 
 enum { OUT_RAW = 0, OUT_U8 = 1, OUT_PLANES = 2 };
 
+// ------------------------------------------------------------------- epilogue
+// One warp handles 32 tensor-memory lanes (= 32 output channels, one per thread)
+// and `cols` accumulator columns starting at tensor-memory address t_row.
+// T(x, t) = #{q : t_q <= x}.  When every |acc| is below 2^24 the count runs on
+// the FP32 pipe (twice the int32 rate): with integer x and t,
+// saturate(float(x) - float(t - 1)) is exactly 1 if x >= t and 0 otherwise;
+// thresholds are clamped to [-2^24 + 1, 2^24] first, which cannot change any
+// comparison with such an accumulator.
+template <int OUT_MODE, int OUT_BITS>
+__device__ __forceinline__ void epilogue_rows(const TcParams &p, uint32_t t_row, int cols, int m, int m0,
+                                              int quad, int lane, int n0) {
+    constexpr int N_THR = (1 << OUT_BITS) - 1;
+    const bool m_ok = m < p.M;
+    int thr_i[N_THR > 0 ? N_THR : 1];
+    float thr_f[N_THR > 0 ? N_THR : 1];
+    if (OUT_MODE != OUT_RAW) {
+#pragma unroll
+        for (int q = 0; q < N_THR; ++q) {
+            const int t = m_ok ? p.thr[(size_t)m * N_THR + q] : 0x7fffffff;
+            thr_i[q] = t;
+            const int tc = t < -16777215 ? -16777215 : (t > 16777216 ? 16777216 : t);
+            thr_f[q] = (float)(tc - 1);
+        }
+    }
+#pragma unroll 1
+    for (int c0 = 0; c0 < cols; c0 += 32) {
+        if (n0 + c0 >= p.N) break;               // warp-uniform: nothing left in this tile
+        int acc[32];
+        tmem_ld32(t_row + c0, acc);
+        if (OUT_MODE == OUT_RAW) {
+            int32_t *o = reinterpret_cast<int32_t *>(p.out);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const int n = n0 + c0 + j;
+                if (m_ok && n < p.N) o[(size_t)n * p.M + m] = acc[j];
+            }
+        } else {
+            int code[32];
+            if (p.fp_count) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const float x = (float)acc[j];
+                    float c = 0.f;
+#pragma unroll
+                    for (int q = 0; q < N_THR; ++q) c += __saturatef(x - thr_f[q]);
+                    code[j] = m_ok ? (int)c : 0;
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    int c = 0;
+#pragma unroll
+                    for (int q = 0; q < N_THR; ++q) c += (acc[j] >= thr_i[q]) ? 1 : 0;
+                    code[j] = m_ok ? c : 0;
+                }
+            }
+            if (OUT_MODE == OUT_U8) {
+                uint8_t *o = reinterpret_cast<uint8_t *>(p.out);
+                if (m < p.ld_out) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int n = n0 + c0 + j;
+                        if (n < p.N) o[(size_t)n * p.ld_out + m] = (uint8_t)code[j];
+                    }
+                }
+            } else {
+                uint32_t keep[OUT_BITS > 0 ? OUT_BITS : 1];
+#pragma unroll
+                for (int b = 0; b < OUT_BITS; ++b) keep[b] = 0;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+#pragma unroll
+                    for (int b = 0; b < OUT_BITS; ++b) {
+                        const uint32_t w = __ballot_sync(0xffffffffu, (code[j] >> b) & 1);
+                        if (lane == j) keep[b] = w;    // lane j keeps column j's word
+                    }
+                }
+                const int mw = (p.M + 31) >> 5, word = (m0 >> 5) + quad, n = n0 + c0 + lane;
+                if (n < p.N && word < mw) {
+#pragma unroll
+                    for (int b = 0; b < OUT_BITS; ++b)
+                        reinterpret_cast<uint32_t *>(p.out)[((size_t)b * p.N + n) * mw + word] = keep[b];
+                }
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------- kernel A: one CTA per tile
 template <int BN, int STAGES>
 struct TcSmem {
     alignas(1024) uint8_t w[STAGES][TC_BM * TC_BK];
@@ -155,7 +246,6 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
     Smem &sm = *reinterpret_cast<Smem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     constexpr uint32_t TMEM_COLS = (2 * BN < 32) ? 32 : 2 * BN;
     constexpr uint32_t STAGE_BYTES = (TC_BM + BN) * TC_BK;
-    constexpr int N_THR = (1 << OUT_BITS) - 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int *abort_flag = &sm.abort_flag;
@@ -230,62 +320,12 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
             const int m0 = (tile % p.tiles_m) * TC_BM, n0 = (tile / p.tiles_m) * BN;
             const uint32_t buf = tcount & 1, acc_ph = (tcount >> 1) & 1;
-            const int m = m0 + quad * 32 + lane;
-            const bool m_ok = m < p.M;
-            int thr_r[N_THR > 0 ? N_THR : 1];
-            if (OUT_MODE != OUT_RAW) {
-#pragma unroll
-                for (int q = 0; q < N_THR; ++q) thr_r[q] = m_ok ? p.thr[(size_t)m * N_THR + q] : 0x7fffffff;
-            }
             ok = mbar_wait(&sm.tmem_full[buf], acc_ph, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * BN;
-#pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                if (n0 + c0 >= p.N) break;               // warp-uniform: nothing left in this tile
-                int acc[32];
-                tmem_ld32(t_row + c0, acc);
-                if (OUT_MODE == OUT_RAW) {
-                    int32_t *o = reinterpret_cast<int32_t *>(p.out);
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int n = n0 + c0 + j;
-                        if (m_ok && n < p.N) o[(size_t)n * p.M + m] = acc[j];
-                    }
-                } else {
-                    uint32_t keep[OUT_BITS > 0 ? OUT_BITS : 1];
-#pragma unroll
-                    for (int b = 0; b < OUT_BITS; ++b) keep[b] = 0;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        int code = 0;
-#pragma unroll
-                        for (int q = 0; q < N_THR; ++q) code += (acc[j] >= thr_r[q]) ? 1 : 0;
-                        if (!m_ok) code = 0;
-                        const int n = n0 + c0 + j;
-                        if (OUT_MODE == OUT_U8) {
-                            if (n < p.N && m < p.ld_out)
-                                reinterpret_cast<uint8_t *>(p.out)[(size_t)n * p.ld_out + m] = (uint8_t)code;
-                        } else {
-#pragma unroll
-                            for (int b = 0; b < OUT_BITS; ++b) {
-                                const uint32_t w = __ballot_sync(0xffffffffu, (code >> b) & 1);
-                                if (lane == j) keep[b] = w;    // lane j keeps column j's word
-                            }
-                        }
-                    }
-                    if (OUT_MODE == OUT_PLANES) {
-                        const int mw = (p.M + 31) >> 5, word = (m0 >> 5) + quad, n = n0 + c0 + lane;
-                        if (n < p.N && word < mw) {
-#pragma unroll
-                            for (int b = 0; b < OUT_BITS; ++b)
-                                reinterpret_cast<uint32_t *>(p.out)[((size_t)b * p.N + n) * mw + word] = keep[b];
-                        }
-                    }
-                }
-            }
+            epilogue_rows<OUT_MODE, OUT_BITS>(p, t_row, BN, m0 + quad * 32 + lane, m0, quad, lane, n0);
             tc_fence_before();
             mbar_arrive(&sm.tmem_empty[buf]);
         }
@@ -296,6 +336,178 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// ---------------------------------------------- kernel B: a CTA pair per 256 x 256 tile
+// Two CTAs of a cluster (two SMs) share one tile: each stages 128 weight rows and
+// 128 of the 256 activation rows, and the leader CTA issues cta_group::2 MMAs
+// (M = 256, N = 256) that read both halves, so each SM pulls 32 KB per 128 depth
+// bytes from L2 instead of 48 KB.  No copy is multicast: each CTA loads only what
+// lands in its own shared memory; its completion bytes are counted on the
+// leader's mbarrier.
+constexpr int T2_STAGES = 6;
+constexpr int T2_BN = 256;
+
+struct Tc2Smem {
+    alignas(1024) uint8_t w[T2_STAGES][TC_BM * TC_BK];
+    alignas(1024) uint8_t a[T2_STAGES][128 * TC_BK];
+    alignas(8) uint64_t full[T2_STAGES];
+    uint64_t empty[T2_STAGES];
+    uint64_t tmem_full[2];
+    uint64_t tmem_empty[2];
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(void *dst, const CUtensorMap *map, uint32_t bar_cluster_addr,
+                                                 int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(bar_cluster_addr), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t *dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)),
+                 "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_i8_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrive on the barrier at cluster address `bar` once all MMAs issued so far are done.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar_cluster_addr) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                 ::"r"(bar_cluster_addr) : "memory");
+}
+
+template <int OUT_MODE, int OUT_BITS>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
+qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a,
+                 const TcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    Tc2Smem &sm = *reinterpret_cast<Tc2Smem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    constexpr uint32_t TMEM_COLS = 2 * T2_BN;
+    constexpr uint32_t PAIR_STAGE_BYTES = 2 * (TC_BM + 128) * TC_BK;   // both CTAs' copies of one stage
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+    volatile int *abort_flag = &sm.abort_flag;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < T2_STAGES; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&sm.tmem_full[b], 1); mbar_init(&sm.tmem_empty[b], 8); }
+        sm.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc_pair(&sm.tmem_base, TMEM_COLS);
+    tc_fence_before();
+    cluster_sync_all();
+    tc_fence_after();
+    const uint32_t tmem_base = sm.tmem_base;
+    const int num_tiles = p.tiles_m * p.tiles_n;       // tiles of 256 x 256
+
+    if (warp == 0) {
+        // ---------------------------------------- producer (one per CTA, own halves)
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+                const int m0 = (tile % p.tiles_m) * 256 + (int)rank * 128;
+                const int n0 = (tile / p.tiles_m) * T2_BN + (int)rank * 128;
+                for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
+                    const int s = it % T2_STAGES;
+                    const uint32_t ph = (it / T2_STAGES) & 1;
+                    if (!(ok = mbar_wait(&sm.empty[s], ph ^ 1, abort_flag))) break;
+                    if (rank == 0) mbar_arrive_expect_tx(&sm.full[s], PAIR_STAGE_BYTES);
+                    const uint32_t leader_full = map_to_cta(smem_u32(&sm.full[s]), 0);
+                    tma_load_2d_pair(sm.w[s], &map_w, leader_full, kb * TC_BK, m0);
+                    tma_load_2d_pair(sm.a[s], &map_a, leader_full, kb * TC_BK, n0);
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ---------------------------------------------- MMA issuer (leader CTA only)
+        if (lane == 0 && rank == 0) {
+            uint32_t it = 0, tcount = 0;
+            bool ok = true;
+            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs, ++tcount) {
+                const uint32_t buf = tcount & 1, acc_ph = (tcount >> 1) & 1;
+                if (!(ok = mbar_wait(&sm.tmem_empty[buf], acc_ph ^ 1, abort_flag))) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * T2_BN;
+                for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
+                    const int s = it % T2_STAGES;
+                    const uint32_t ph = (it / T2_STAGES) & 1;
+                    if (!(ok = mbar_wait(&sm.full[s], ph, abort_flag))) break;
+                    tc_fence_after();
+                    const uint64_t dw = umma_smem_desc(smem_u32(sm.w[s]));
+                    const uint64_t da = umma_smem_desc(smem_u32(sm.a[s]));
+#pragma unroll
+                    for (int kk = 0; kk < TC_BK / 32; ++kk)
+                        umma_i8_pair(d_tmem, dw + 2 * kk, da + 2 * kk, p.idesc, (kb | kk) != 0);
+                    // free the stage in both CTAs
+                    umma_commit_pair(map_to_cta(smem_u32(&sm.empty[s]), 0));
+                    umma_commit_pair(map_to_cta(smem_u32(&sm.empty[s]), 1));
+                }
+                if (ok) {
+                    umma_commit_pair(map_to_cta(smem_u32(&sm.tmem_full[buf]), 0));
+                    umma_commit_pair(map_to_cta(smem_u32(&sm.tmem_full[buf]), 1));
+                }
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------- epilogue (each CTA: its 128 rows)
+        const int quad = warp & 3;
+        uint32_t tcount = 0;
+        bool ok = true;
+        for (int tile = pair; ok && tile < num_tiles; tile += num_pairs, ++tcount) {
+            const int m0 = (tile % p.tiles_m) * 256 + (int)rank * 128, n0 = (tile / p.tiles_m) * T2_BN;
+            const uint32_t buf = tcount & 1, acc_ph = (tcount >> 1) & 1;
+            ok = mbar_wait(&sm.tmem_full[buf], acc_ph, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * T2_BN;
+            epilogue_rows<OUT_MODE, OUT_BITS>(p, t_row, T2_BN, m0 + quad * 32 + lane, m0, quad, lane, n0);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&sm.tmem_empty[buf]), 0));
+        }
+    }
+
+    // the peer may still read this CTA's shared memory or signal its barriers
+    tc_fence_before();
+    cluster_sync_all();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, TMEM_COLS);
     }
 }
 
@@ -347,43 +559,100 @@ static qnn_status launch_cfg(const CUtensorMap &mw, const CUtensorMap &ma, const
     return launch_status();
 }
 
+template <int OUT_MODE, int OUT_BITS>
+static qnn_status launch_pair_cfg(const CUtensorMap &mw, const CUtensorMap &ma, const TcParams &p, cudaStream_t s) {
+    auto kern = qgemm_tc2_kernel<OUT_MODE, OUT_BITS>;
+    const size_t smem = sizeof(Tc2Smem) + 1024;
+    static bool attr_done = false;
+    if (!attr_done) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return QNN_ERR_CUDA;
+        attr_done = true;
+    }
+    const int tiles = p.tiles_m * p.tiles_n;
+    const int max_pairs = sm_count() / 2;
+    const int pairs = tiles < max_pairs ? tiles : max_pairs;
+    kern<<<2 * pairs, TC_THREADS, smem, s>>>(mw, ma, p);
+    count_launch();
+    return launch_status();
+}
+
+#define QNN_TC_DISPATCH(CALL_RAW, CALL)                                                    \
+    if (mode == OUT_RAW) return CALL_RAW;                                                  \
+    switch (out_bits) {                                                                    \
+        case 1: return mode == OUT_U8 ? CALL(OUT_U8, 1) : CALL(OUT_PLANES, 1);             \
+        case 2: return mode == OUT_U8 ? CALL(OUT_U8, 2) : CALL(OUT_PLANES, 2);             \
+        case 3: return mode == OUT_U8 ? CALL(OUT_U8, 3) : CALL(OUT_PLANES, 3);             \
+        case 4: return mode == OUT_U8 ? CALL(OUT_U8, 4) : CALL(OUT_PLANES, 4);             \
+    }                                                                                      \
+    return QNN_ERR_UNSUPPORTED;
+
 template <int BN, int STAGES>
 static qnn_status launch_out(int mode, int out_bits, const CUtensorMap &mw, const CUtensorMap &ma,
                              const TcParams &p, cudaStream_t s) {
-    if (mode == OUT_RAW) return launch_cfg<BN, STAGES, OUT_RAW, 0>(mw, ma, p, s);
-#define QNN_TC_CASE(B_)                                                                   \
-    if (out_bits == B_)                                                                   \
-        return mode == OUT_U8 ? launch_cfg<BN, STAGES, OUT_U8, B_>(mw, ma, p, s)         \
-                              : launch_cfg<BN, STAGES, OUT_PLANES, B_>(mw, ma, p, s);
-    QNN_TC_CASE(1) QNN_TC_CASE(2) QNN_TC_CASE(3) QNN_TC_CASE(4)
-#undef QNN_TC_CASE
-    return QNN_ERR_UNSUPPORTED;
+#define QNN_C1(MODE_, BITS_) launch_cfg<BN, STAGES, MODE_, BITS_>(mw, ma, p, s)
+    QNN_TC_DISPATCH(QNN_C1(OUT_RAW, 0), QNN_C1)
+#undef QNN_C1
+}
+
+static qnn_status launch_pair_out(int mode, int out_bits, const CUtensorMap &mw, const CUtensorMap &ma,
+                                  const TcParams &p, cudaStream_t s) {
+#define QNN_C2(MODE_, BITS_) launch_pair_cfg<MODE_, BITS_>(mw, ma, p, s)
+    QNN_TC_DISPATCH(QNN_C2(OUT_RAW, 0), QNN_C2)
+#undef QNN_C2
+}
+
+// Kernel choice.  QNN_TC_KERNEL=single|pair in the environment overrides it (tests, sweeps).
+static bool choose_pair_kernel(const qnn_gemm_desc *d, int sms) {
+    const char *force = getenv("QNN_TC_KERNEL");
+    if (force && force[0] == 's') return false;
+    if (force && force[0] == 'p') return true;
+    if (d->N < 256 || d->M <= 128) return false;
+    // estimated time in units of 128x256-tile main loops; a pair tile runs ~0.75 of two of those
+    const long long t1 = (long long)ceil_div(d->M, 128) * ceil_div(d->N, 256);
+    const long long t2 = (long long)ceil_div(d->M, 256) * ceil_div(d->N, 256);
+    const double cost1 = (double)ceil_div((int)t1, sms);
+    const double cost2 = 0.75 * (double)ceil_div((int)t2, sms / 2);
+    return t1 >= sms && cost2 < cost1;
 }
 
 qnn_status gemm_tc_launch(const qnn_gemm_desc *d, const void *W, const void *A, const int32_t *thr,
                           void *out, cudaStream_t s) {
     const int ld = round_up(d->K, 16);
-    // column tile: the widest that still gives every SM a tile
     const int sms = sm_count();
+    const bool pair = choose_pair_kernel(d, sms);
+
+    TcParams p;
+    p.thr = thr; p.out = out; p.M = d->M; p.N = d->N; p.K = d->K;
+    p.num_kb = ceil_div(d->K, TC_BK);
+    p.ld_out = round_up(d->M, 16);
+    const double wmax = d->w_enc == QNN_ENC_BIPOLAR ? 1.0
+                        : (d->w_enc == QNN_ENC_SIGNED ? double(1 << (d->w_bits - 1)) : double((1 << d->w_bits) - 1));
+    const double amax = d->a_enc == QNN_ENC_BIPOLAR ? 1.0
+                        : (d->a_enc == QNN_ENC_SIGNED ? double(1 << (d->a_bits - 1)) : double((1 << d->a_bits) - 1));
+    p.fp_count = (double(d->K) * wmax * amax < 16777216.0) ? 1 : 0;
+    const uint32_t w_s8 = d->w_enc == QNN_ENC_UNSIGNED ? 0u : 1u;
+    const uint32_t a_s8 = d->a_enc == QNN_ENC_UNSIGNED ? 0u : 1u;
+    const uint32_t idesc_base = (2u << 4)      // accumulator format: s32
+                                | (w_s8 << 7)  // A-operand (weights) format: 0 = u8, 1 = s8
+                                | (a_s8 << 10);   // B-operand (activations) format; both K-major
+    const int mode = !thr ? OUT_RAW : (d->out_fmt == QNN_FMT_INT8 ? OUT_U8 : OUT_PLANES);
+    CUtensorMap mw, ma;
+
+    if (pair) {
+        if (!make_map(&mw, W, d->M, d->K, ld, TC_BM) || !make_map(&ma, A, d->N, d->K, ld, 128)) return QNN_ERR_CUDA;
+        p.tiles_m = ceil_div(d->M, 256); p.tiles_n = ceil_div(d->N, T2_BN);
+        p.idesc = idesc_base | ((uint32_t)(T2_BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+        return launch_pair_out(mode, d->out_bits, mw, ma, p, s);
+    }
+    // column tile: the widest that still gives every SM a tile
     const int tiles_m = ceil_div(d->M, TC_BM);
     int bn = 256;
     while (bn > 32 && (long long)tiles_m * ceil_div(d->N, bn) < sms) bn >>= 1;
     if (bn == 64) bn = 32;
-
-    CUtensorMap mw, ma;
     if (!make_map(&mw, W, d->M, d->K, ld, TC_BM) || !make_map(&ma, A, d->N, d->K, ld, bn)) return QNN_ERR_CUDA;
-
-    TcParams p;
-    p.thr = thr; p.out = out; p.M = d->M; p.N = d->N; p.K = d->K;
-    p.tiles_m = tiles_m; p.tiles_n = ceil_div(d->N, bn); p.num_kb = ceil_div(d->K, TC_BK);
-    p.ld_out = round_up(d->M, 16);
-    const uint32_t w_s8 = d->w_enc == QNN_ENC_UNSIGNED ? 0u : 1u;
-    const uint32_t a_s8 = d->a_enc == QNN_ENC_UNSIGNED ? 0u : 1u;
-    p.idesc = (2u << 4)                 // accumulator format: s32
-              | (w_s8 << 7)             // A-operand (weights) format: 0 = u8, 1 = s8
-              | (a_s8 << 10)            // B-operand (activations) format
-              | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);   // both K-major
-    const int mode = !thr ? OUT_RAW : (d->out_fmt == QNN_FMT_INT8 ? OUT_U8 : OUT_PLANES);
+    p.tiles_m = tiles_m; p.tiles_n = ceil_div(d->N, bn);
+    p.idesc = idesc_base | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
     switch (bn) {
         case 256: return launch_out<256, 4>(mode, d->out_bits, mw, ma, p, s);
         case 128: return launch_out<128, 6>(mode, d->out_bits, mw, ma, p, s);

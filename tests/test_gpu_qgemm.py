@@ -134,3 +134,65 @@ def test_outputs_monotone_in_accumulator(qb):
     for m in range(0, 256, 17):
         order = np.argsort(acc[:, m], kind="stable")
         assert np.all(np.diff(codes[order, m].astype(np.int32)) >= 0)
+
+
+@pytest.fixture
+def force_tc_kernel(monkeypatch):
+    def _set(which):
+        monkeypatch.setenv("QNN_TC_KERNEL", which)
+    return _set
+
+
+@pytest.mark.parametrize("which", ["single", "pair"])
+@pytest.mark.parametrize("M,N,K,w,a", [
+    (64, 256, 576, 1, 2), (197, 301, 1100, 2, 2), (512, 768, 2048, 1, 2), (300, 1000, 4100, 4, 4),
+    (256, 256, 128, 3, 3), (1, 1, 1, 2, 2), (129, 257, 129, 2, 3), (640, 520, 16, 4, 1),
+])
+def test_both_tensor_core_kernels(qb, force_tc_kernel, which, M, N, K, w, a):
+    """The one-CTA and the CTA-pair (cta_group::2) kernels on the same problems,
+    every output mode, incl. sizes with ragged M/N/K tails and fewer tiles than SMs."""
+    force_tc_kernel(which)
+    case = synth.gemm_case(1000 + M + N + K, M, N, K, w, a)
+    run_case(qb, case, INT8, INT8)
+    run_case(qb, case, INT8, BITPLANES)
+    run_case(qb, case, INT8, INT8, raw=True)
+
+
+@pytest.mark.parametrize("which", ["single", "pair"])
+def test_integer_count_path_for_large_accumulators(qb, force_tc_kernel, which):
+    """8-bit x 8-bit with K large enough that |acc| can exceed 2^24: the epilogue must
+    count thresholds in integer arithmetic; thresholds beyond +-2^24 included."""
+    force_tc_kernel(which)
+    case = synth.gemm_case(1100, 200, 300, 1024, 8, 8, synth.SIGNED, synth.UNSIGNED, out_bits=3)
+    case.thr[0] = [-(2**31), -(2**24) - 5, -(2**24), 0, 2**24, 2**24 + 7, 2**31 - 1]
+    run_case(qb, case, INT8, INT8)
+    small = synth.gemm_case(1101, 200, 300, 512, 4, 4, out_bits=3)
+    small.thr[0] = [-(2**31), -(2**24) - 5, -(2**24), 0, 2**24, 2**24 + 7, 2**31 - 1]
+    small.thr[1] = [-16777215, -16777214, -1, 0, 1, 16777215, 16777216]
+    run_case(qb, small, INT8, INT8)
+    run_case(qb, small, BITPLANES, INT8)
+
+
+@pytest.mark.parametrize("w,a", [(1, 2), (4, 4)])
+def test_full_size_4096_sampled(qb, w, a):
+    """The benchmark's problem size and launch configuration (M=N=K=4096), checked on
+    sampled outputs the oracle computes one by one, plus whole rows/columns."""
+    case = synth.gemm_case(2000 + 10 * w + a, 4096, 4096, 4096, w, a)
+    Wd = qb.to_device_logical(case.W, case.w_enc)
+    Ad = qb.to_device_logical(case.At, case.a_enc)
+    Wp, Ap = qb.pack(Wd, w, case.w_enc, INT8), qb.pack(Ad, a, case.a_enc, INT8)
+    d = qb.gemm_desc(4096, 4096, 4096, w, a, a, case.w_enc, case.a_enc, INT8, INT8)
+    codes = qb.qgemm(d, Wp, Ap, torch.from_numpy(case.thr).cuda()).cpu().numpy().reshape(4096, 4096)
+    raw = qb.qgemm(d, Wp, Ap, None).cpu().numpy()
+    rng = np.random.default_rng(7)
+    rows = np.concatenate([rng.integers(0, 4096, 3000), [0, 4095, 127, 128, 255, 256, 4095]])
+    cols = np.concatenate([rng.integers(0, 4096, 3000), [0, 4095, 255, 256, 4095, 0, 0]])
+    acc = orc.dot_at(case.W, case.At, rows, cols)
+    assert np.array_equal(raw[cols, rows].astype(np.int64), acc)
+    want = (acc[:, None] >= case.thr[rows]).sum(axis=1)
+    assert np.array_equal(codes[cols, rows].astype(np.int64), want)
+    # one full weight row and one full column through the oracle GEMM
+    full_row = orc.qgemm(case.W[777:778], case.At, case.thr[777:778])[0]
+    assert np.array_equal(codes[:, 777].astype(np.int64), full_row)
+    full_col = orc.qgemm(case.W, case.At[1234:1235], case.thr)[:, 0]
+    assert np.array_equal(codes[1234, :].astype(np.int64), full_col)
