@@ -7,16 +7,21 @@
 // Section 3.1 equals.  The epilogue applies T(x, t) of Section 2.1.1 to the
 // accumulators straight out of tensor memory, so they never reach HBM.
 //
-// Kernel structure (persistent, one CTA per SM, 192 threads):
-//   warp 0     TMA producer: 128-byte-swizzled K-major tiles of W (128 rows)
-//              and A (BN rows) into a STAGES-deep shared-memory ring
+// Orientation: activation rows (pixels, the GEMM's N) are the MMA's M side and
+// land on the 128 tensor-memory lanes; weight rows (output channels, the GEMM's
+// M) are the MMA's N side and land on tensor-memory columns.  An epilogue thread
+// therefore owns one pixel and reads 32 consecutive channels per tcgen05.ld,
+// which is exactly the channels-fastest output layout: 32 codes leave as two
+// 16-byte stores, and the 32 bits of one plane are one word of the
+// channel-interleaved layout of Section 3.2.
+//
+// Kernel structure (persistent, one CTA per SM, 320 threads):
+//   warp 0     TMA producer: 128-byte-swizzled K-major tiles of the activations
+//              (128 rows) and weights (BN rows) into a shared-memory ring
 //   warp 1     allocates tensor memory; one lane issues the MMAs
 //              (M = 128, N = BN, K = 32 per instruction) and commits to mbarriers
-//   warps 2-5  epilogue: tcgen05.ld of a 32-lane x 32-column block, threshold
-//              count with the row's thresholds in registers, store.
-// Output channels (weight rows) lie on the 128 tensor-memory lanes, so each
-// epilogue thread owns one channel, and a warp ballot over code bits yields one
-// word of the channel-interleaved bit-plane layout of Section 3.2.
+//   warps 2-9  epilogue: warp e reads lanes 32*(e%4).. and the column half e/4;
+//              thresholds of the tile's channels are staged in shared memory.
 // Two accumulator buffers in tensor memory let the epilogue of tile t overlap the
 // main loop of tile t+1.  Every wait is bounded; on expiry the CTA records
 // QNN_ERR_DEVICE_TIMEOUT in the device status word, drains and exits.
@@ -29,9 +34,16 @@ namespace qnn {
 
 __device__ int g_dev_status;   // QNN_OK or QNN_ERR_DEVICE_TIMEOUT
 
-constexpr int TC_BM = 128;          // weight rows per tile = tensor-memory lanes
+#ifdef QNN_TC_TRACE
+// Debug builds only: per-tile clock64() stamps of CTA 0, [slot][tile round].
+__device__ long long g_trace[16 * 512];
+#define QNN_TRACE(slot, idx) do { if (blockIdx.x == 0 && (idx) < 512) g_trace[(slot) * 512 + (idx)] = clock64(); } while (0)
+#else
+#define QNN_TRACE(slot, idx) do { } while (0)
+#endif
+
+constexpr int TC_BP = 128;          // activation rows (pixels) per tile = tensor-memory lanes
 constexpr int TC_BK = 128;          // depth bytes per stage = one 128B swizzle row
-constexpr int TC_THREADS = 192;
 constexpr long long TC_WAIT_CYCLES = 2000000000ll;   // ~1 s
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -99,19 +111,6 @@ __device__ __forceinline__ void umma_commit(uint64_t *bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                  : "memory");
 }
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, int (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n\t"
-        "tcgen05.wait::ld.sync.aligned;"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-}
-
 // K-major operand tile, rows at a 128-byte pitch, 128B swizzle (what TMA writes
 // with CU_TENSOR_MAP_SWIZZLE_128B): 8-row groups are 1024 bytes apart.
 __device__ __forceinline__ uint64_t umma_smem_desc(uint32_t saddr) {
@@ -127,132 +126,261 @@ __device__ __forceinline__ uint64_t umma_smem_desc(uint32_t saddr) {
 struct TcParams {
     const int32_t *thr;    // [M][n_thr] or null
     void *out;
-    int M, N, K;
-    int tiles_m, tiles_n, num_kb;
+    int M, N, K;           // channels (weight rows), pixels (activation rows), depth
+    int tiles_p, tiles_c, num_kb;
     int ld_out;            // INT8 output row pitch
-    int fp_count;          // 1: |acc| < 2^24, thresholds are counted on the FP32 pipe
+    int fp_count;          // 1: |acc| < 2^22, thresholds are counted on the FP32 pipe
     uint32_t idesc;
 };
 
 enum { OUT_RAW = 0, OUT_U8 = 1, OUT_PLANES = 2 };
 
 // ------------------------------------------------------------------- epilogue
-// One warp handles 32 tensor-memory lanes (= 32 output channels, one per thread)
-// and `cols` accumulator columns starting at tensor-memory address t_row.
-// T(x, t) = #{q : t_q <= x}.  When every |acc| is below 2^24 the count runs on
-// the FP32 pipe (twice the int32 rate): with integer x and t,
-// saturate(float(x) - float(t - 1)) is exactly 1 if x >= t and 0 otherwise;
-// thresholds are clamped to [-2^24 + 1, 2^24] first, which cannot change any
-// comparison with such an accumulator.
+// T(x, t) = #{q : t_q <= x}.  When every |acc| is below 2^22 the count runs on the
+// FP32 pipe (twice the int32 rate, no conversions): the int32 accumulator x is
+// turned into the float 1.5*2^23 + x by one integer add on its bit pattern, each
+// threshold is held as the float 1.5*2^23 + (t - 1), and for integers
+// saturate((1.5*2^23 + x) - (1.5*2^23 + t - 1)) is exactly 1 if x >= t, else 0.
+// Thresholds are clamped to [-2^22 + 1, 2^22] first, which cannot change a
+// comparison with such an accumulator.  Counts of two neighbouring channels are
+// accumulated in one float on top of 1.5*2^23 (the second scaled by 256), so the
+// two codes are the low two bytes of the sum's bit pattern.
+constexpr int EPI_WARPS = 8;
+constexpr int TC_THREADS = 64 + 32 * EPI_WARPS;
+constexpr float FP_MAGIC = 12582912.0f;        // 1.5 * 2^23, bit pattern 0x4B400000
+constexpr int FP_MAGIC_BITS = 0x4B400000;
+constexpr int FP_LIMIT = 1 << 22;
+
+// thresholds per channel in shared memory, padded to a multiple of four
+__host__ __device__ constexpr int thr_slots(int out_bits) {
+    return out_bits <= 0 ? 4 : (((1 << out_bits) - 1 + 3) / 4 * 4);
+}
+
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, int (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+// Completes every tcgen05.ld issued so far; the registers pass through the statement so
+// that no use of them can be scheduled ahead of it.
+__device__ __forceinline__ void tmem_ld_wait(int (&r)[32]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+        : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+          "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+          "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+          "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+        :: "memory");
+}
+
+// Bits b, 8+b, 16+b, 24+b of x gathered into the low nibble.
+__device__ __forceinline__ uint32_t nibble_of_plane(uint32_t x, int b) {
+    return (((x >> b) & 0x01010101u) * 0x01020408u) >> 24;
+}
+
+// Stage the thresholds of channels [c0, c0 + bn) in shared memory: float form for the
+// FP count, raw int32 otherwise; slots past the row's thresholds and channels past M
+// hold a value no accumulator reaches.
+template <int OUT_BITS>
+__device__ __forceinline__ void stage_thresholds(const TcParams &p, int *thr_s, int c0, int bn, int etid) {
+    constexpr int N_THR = (1 << OUT_BITS) - 1, NT = thr_slots(OUT_BITS);
+    for (int idx = etid; idx < bn * NT; idx += 32 * EPI_WARPS) {
+        const int c = idx / NT, q = idx - c * NT, m = c0 + c;
+        int t = 0x7fffffff;
+        if (q < N_THR && m < p.M) t = p.thr[(size_t)m * N_THR + q];
+        if (p.fp_count) {
+            const int tc = t <= -FP_LIMIT ? -FP_LIMIT + 1 : (t > FP_LIMIT ? FP_LIMIT : t);
+            t = FP_MAGIC_BITS + (tc - 1);
+        }
+        thr_s[idx] = t;
+    }
+}
+
+// One chunk: this thread's pixel n, channels mc .. mc+31 (accumulators acc[0..31]).
 template <int OUT_MODE, int OUT_BITS>
-__device__ __forceinline__ void epilogue_rows(const TcParams &p, uint32_t t_row, int cols, int m, int m0,
-                                              int quad, int lane, int n0) {
-    constexpr int N_THR = (1 << OUT_BITS) - 1;
-    const bool m_ok = m < p.M;
-    int thr_i[N_THR > 0 ? N_THR : 1];
-    float thr_f[N_THR > 0 ? N_THR : 1];
-    if (OUT_MODE != OUT_RAW) {
+__device__ __forceinline__ void epilogue_chunk(const TcParams &p, const int *thr_c, const int (&acc)[32],
+                                               int n, bool n_ok, int mc) {
+    constexpr int N_THR = (1 << OUT_BITS) - 1, NT = thr_slots(OUT_BITS);
+    if (OUT_MODE == OUT_RAW) {
+        if (!n_ok) return;
+        int32_t *o = reinterpret_cast<int32_t *>(p.out) + (size_t)n * p.M + mc;
+        if ((p.M & 3) == 0 && mc + 32 <= p.M) {
 #pragma unroll
-        for (int q = 0; q < N_THR; ++q) {
-            const int t = m_ok ? p.thr[(size_t)m * N_THR + q] : 0x7fffffff;
-            thr_i[q] = t;
-            const int tc = t < -16777215 ? -16777215 : (t > 16777216 ? 16777216 : t);
-            thr_f[q] = (float)(tc - 1);
+            for (int v = 0; v < 8; ++v)
+                reinterpret_cast<int4 *>(o)[v] = make_int4(acc[4 * v], acc[4 * v + 1], acc[4 * v + 2], acc[4 * v + 3]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (mc + j < p.M) o[j] = acc[j];
+        }
+        return;
+    }
+    uint32_t packed[8];                          // four codes per word, one byte each
+    if (p.fp_count) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            uint32_t pr[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int j = 4 * k + 2 * h;
+                const float x0 = __int_as_float(acc[j] + FP_MAGIC_BITS);
+                const float x1 = __int_as_float(acc[j + 1] + FP_MAGIC_BITS);
+                float c = FP_MAGIC;
+#pragma unroll
+                for (int v = 0; v < NT / 4; ++v) {
+                    const float4 t0 = *reinterpret_cast<const float4 *>(thr_c + j * NT + 4 * v);
+                    const float4 t1 = *reinterpret_cast<const float4 *>(thr_c + (j + 1) * NT + 4 * v);
+                    if (4 * v + 0 < N_THR) { c += __saturatef(x0 - t0.x); c = fmaf(__saturatef(x1 - t1.x), 256.f, c); }
+                    if (4 * v + 1 < N_THR) { c += __saturatef(x0 - t0.y); c = fmaf(__saturatef(x1 - t1.y), 256.f, c); }
+                    if (4 * v + 2 < N_THR) { c += __saturatef(x0 - t0.z); c = fmaf(__saturatef(x1 - t1.z), 256.f, c); }
+                    if (4 * v + 3 < N_THR) { c += __saturatef(x0 - t0.w); c = fmaf(__saturatef(x1 - t1.w), 256.f, c); }
+                }
+                pr[h] = (uint32_t)__float_as_int(c);
+            }
+            packed[k] = __byte_perm(pr[0], pr[1], 0x5410);
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            uint32_t w = 0;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int j = 4 * k + e;
+                int c = 0;
+#pragma unroll
+                for (int q = 0; q < N_THR; ++q) c += (acc[j] >= thr_c[j * NT + q]) ? 1 : 0;
+                w |= (uint32_t)c << (8 * e);
+            }
+            packed[k] = w;
         }
     }
-#pragma unroll 1
-    for (int c0 = 0; c0 < cols; c0 += 32) {
-        if (n0 + c0 >= p.N) break;               // warp-uniform: nothing left in this tile
-        int acc[32];
-        tmem_ld32(t_row + c0, acc);
-        if (OUT_MODE == OUT_RAW) {
-            int32_t *o = reinterpret_cast<int32_t *>(p.out);
+    if (!n_ok) return;
+    if (OUT_MODE == OUT_U8) {
+        uint8_t *o = reinterpret_cast<uint8_t *>(p.out) + (size_t)n * p.ld_out + mc;
+        const int valid = p.ld_out - mc;         // a multiple of 16
+        if (valid >= 16) reinterpret_cast<uint4 *>(o)[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+        if (valid >= 32) reinterpret_cast<uint4 *>(o)[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+    } else {
+        const int mw = (p.M + 31) >> 5, word = mc >> 5;
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const int n = n0 + c0 + j;
-                if (m_ok && n < p.N) o[(size_t)n * p.M + m] = acc[j];
-            }
-        } else {
-            int code[32];
-            if (p.fp_count) {
+        for (int b = 0; b < OUT_BITS; ++b) {
+            uint32_t bits = 0;
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const float x = (float)acc[j];
-                    float c = 0.f;
-#pragma unroll
-                    for (int q = 0; q < N_THR; ++q) c += __saturatef(x - thr_f[q]);
-                    code[j] = m_ok ? (int)c : 0;
-                }
-            } else {
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    int c = 0;
-#pragma unroll
-                    for (int q = 0; q < N_THR; ++q) c += (acc[j] >= thr_i[q]) ? 1 : 0;
-                    code[j] = m_ok ? c : 0;
-                }
-            }
-            if (OUT_MODE == OUT_U8) {
-                uint8_t *o = reinterpret_cast<uint8_t *>(p.out);
-                if (m < p.ld_out) {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int n = n0 + c0 + j;
-                        if (n < p.N) o[(size_t)n * p.ld_out + m] = (uint8_t)code[j];
-                    }
-                }
-            } else {
-                uint32_t keep[OUT_BITS > 0 ? OUT_BITS : 1];
-#pragma unroll
-                for (int b = 0; b < OUT_BITS; ++b) keep[b] = 0;
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-#pragma unroll
-                    for (int b = 0; b < OUT_BITS; ++b) {
-                        const uint32_t w = __ballot_sync(0xffffffffu, (code[j] >> b) & 1);
-                        if (lane == j) keep[b] = w;    // lane j keeps column j's word
-                    }
-                }
-                const int mw = (p.M + 31) >> 5, word = (m0 >> 5) + quad, n = n0 + c0 + lane;
-                if (n < p.N && word < mw) {
-#pragma unroll
-                    for (int b = 0; b < OUT_BITS; ++b)
-                        reinterpret_cast<uint32_t *>(p.out)[((size_t)b * p.N + n) * mw + word] = keep[b];
-                }
-            }
+            for (int k = 0; k < 8; ++k) bits |= nibble_of_plane(packed[k], b) << (4 * k);
+            reinterpret_cast<uint32_t *>(p.out)[((size_t)b * p.N + n) * mw + word] = bits;
         }
     }
 }
 
+// Columns [c_begin, c_end) of one accumulator tile for this thread's pixel.  The
+// tensor-memory load of the next chunk is in flight while the current one is processed.
+template <int OUT_MODE, int OUT_BITS>
+__device__ __forceinline__ void epilogue_cols(const TcParams &p, const int *thr_s, uint32_t t_row,
+                                              int c_begin, int c_end, int n, int m0) {
+    constexpr int NT = thr_slots(OUT_BITS);
+    int c_stop = c_end;                                  // skip chunks wholly beyond M (warp-uniform)
+    if (m0 + c_stop > p.M) c_stop = c_begin + ((p.M - m0 - c_begin + 31) & ~31);
+    if (c_begin >= c_stop) return;
+    const bool n_ok = n < p.N;
+    int acc_a[32], acc_b[32];
+    tmem_ld32_issue(t_row + c_begin, acc_a);
+#pragma unroll 1
+    for (int c0 = c_begin; c0 < c_stop; c0 += 64) {
+        tmem_ld_wait(acc_a);
+        const bool has_b = c0 + 32 < c_stop;
+        if (has_b) tmem_ld32_issue(t_row + c0 + 32, acc_b);
+        epilogue_chunk<OUT_MODE, OUT_BITS>(p, thr_s + c0 * NT, acc_a, n, n_ok, m0 + c0);
+        if (has_b) {
+            tmem_ld_wait(acc_b);
+            if (c0 + 64 < c_stop) tmem_ld32_issue(t_row + c0 + 64, acc_a);
+            epilogue_chunk<OUT_MODE, OUT_BITS>(p, thr_s + (c0 + 32) * NT, acc_b, n, n_ok, m0 + c0 + 32);
+        }
+    }
+}
+
+// Epilogue warps meet on an mbarrier (bounded wait) instead of a named barrier.
+__device__ __forceinline__ bool epi_sync(uint64_t *bar, uint32_t parity, int lane, volatile int *abort_flag) {
+    __syncwarp();
+    bool ok = true;
+    if (lane == 0) {
+        mbar_arrive(bar);
+        ok = mbar_wait(bar, parity, abort_flag);
+    }
+    return __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+}
+
+// Per-tile epilogue shared by both kernels.  Returns false if a wait ran out.
+template <int OUT_MODE, int OUT_BITS>
+__device__ __forceinline__ bool epilogue_tile(const TcParams &p, int *thr_s, uint64_t *thr_bar, int &staged_c0,
+                                              uint32_t &refills, uint64_t *tmem_full, uint32_t full_parity,
+                                              uint32_t t_acc, int bn, int p0, int c0, int warp, int lane,
+                                              volatile int *abort_flag, int full_parity_dbg = 0) {
+    const int quad = warp & 3, half = (warp - 2) >> 2;
+    const bool tr = warp == 2 && lane == 0;
+    if (tr) QNN_TRACE(0, full_parity_dbg);
+    if (OUT_MODE != OUT_RAW && staged_c0 != c0) {
+        // everyone is done with the old thresholds -> refill -> everyone sees the new ones
+        if (!epi_sync(&thr_bar[0], refills & 1, lane, abort_flag)) return false;
+        stage_thresholds<OUT_BITS>(p, thr_s, c0, bn, (warp - 2) * 32 + lane);
+        if (!epi_sync(&thr_bar[1], refills & 1, lane, abort_flag)) return false;
+        ++refills;
+        staged_c0 = c0;
+    }
+    bool ok = true;
+    if (tr) QNN_TRACE(1, full_parity_dbg);
+    if (lane == 0) ok = mbar_wait(tmem_full, full_parity, abort_flag);    // one lane polls
+    if (__shfl_sync(0xffffffffu, (int)ok, 0) == 0) return false;
+    if (tr) QNN_TRACE(2, full_parity_dbg);
+    tc_fence_after();
+    const int hcols = bn >= 64 ? bn / 2 : bn;
+    const int c_begin = half * hcols, c_end = (bn >= 64 || half == 0) ? c_begin + hcols : c_begin;
+    epilogue_cols<OUT_MODE, OUT_BITS>(p, thr_s, t_acc + ((uint32_t)(quad * 32) << 16), c_begin, c_end,
+                                      p0 + quad * 32 + lane, c0);
+    tc_fence_before();
+    __syncwarp();
+    if (tr) QNN_TRACE(3, full_parity_dbg);
+    return true;
+}
+
 // ------------------------------------------------------- kernel A: one CTA per tile
-template <int BN, int STAGES>
+template <int BN, int STAGES, int OUT_BITS>
 struct TcSmem {
-    alignas(1024) uint8_t w[STAGES][TC_BM * TC_BK];
-    alignas(1024) uint8_t a[STAGES][BN * TC_BK];
+    alignas(1024) uint8_t act[STAGES][TC_BP * TC_BK];
+    alignas(1024) uint8_t wgt[STAGES][BN * TC_BK];
+    alignas(16) int thr[BN * thr_slots(OUT_BITS)];
     alignas(8) uint64_t full[STAGES];
     uint64_t empty[STAGES];
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
+    uint64_t thr_bar[2];
     uint32_t tmem_base;
     int abort_flag;
 };
 
 template <int BN, int STAGES, int OUT_MODE, int OUT_BITS>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a,
+qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_constant__ CUtensorMap map_wgt,
                 const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
-    using Smem = TcSmem<BN, STAGES>;
+    using Smem = TcSmem<BN, STAGES, OUT_BITS>;
     Smem &sm = *reinterpret_cast<Smem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     constexpr uint32_t TMEM_COLS = (2 * BN < 32) ? 32 : 2 * BN;
-    constexpr uint32_t STAGE_BYTES = (TC_BM + BN) * TC_BK;
+    constexpr uint32_t STAGE_BYTES = (TC_BP + BN) * TC_BK;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int *abort_flag = &sm.abort_flag;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&sm.tmem_full[b], 1); mbar_init(&sm.tmem_empty[b], 128); }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&sm.tmem_full[b], 1); mbar_init(&sm.tmem_empty[b], EPI_WARPS);
+            mbar_init(&sm.thr_bar[b], EPI_WARPS);
+        }
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -261,7 +389,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = sm.tmem_base;
-    const int num_tiles = p.tiles_m * p.tiles_n;
+    const int num_tiles = p.tiles_p * p.tiles_c;
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
@@ -269,14 +397,14 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
             uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-                const int m0 = (tile % p.tiles_m) * TC_BM, n0 = (tile / p.tiles_m) * BN;
+                const int p0 = (tile % p.tiles_p) * TC_BP, c0 = (tile / p.tiles_p) * BN;
                 for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1;
                     if (!(ok = mbar_wait(&sm.empty[s], ph ^ 1, abort_flag))) break;
                     mbar_arrive_expect_tx(&sm.full[s], STAGE_BYTES);
-                    tma_load_2d(sm.w[s], &map_w, &sm.full[s], kb * TC_BK, m0);
-                    tma_load_2d(sm.a[s], &map_a, &sm.full[s], kb * TC_BK, n0);
+                    tma_load_2d(sm.act[s], &map_act, &sm.full[s], kb * TC_BK, p0);
+                    tma_load_2d(sm.wgt[s], &map_wgt, &sm.full[s], kb * TC_BK, c0);
                 }
             }
             if (!ok) {
@@ -301,11 +429,11 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
                     const uint32_t ph = (it / STAGES) & 1;
                     if (!(ok = mbar_wait(&sm.full[s], ph, abort_flag))) break;
                     tc_fence_after();
-                    const uint64_t dw = umma_smem_desc(smem_u32(sm.w[s]));
-                    const uint64_t da = umma_smem_desc(smem_u32(sm.a[s]));
+                    const uint64_t da = umma_smem_desc(smem_u32(sm.act[s]));
+                    const uint64_t db = umma_smem_desc(smem_u32(sm.wgt[s]));
 #pragma unroll
                     for (int kk = 0; kk < TC_BK / 32; ++kk)   // 32 depth bytes per MMA: +2 in 16-byte units
-                        umma_i8(d_tmem, dw + 2 * kk, da + 2 * kk, p.idesc, (kb | kk) != 0);
+                        umma_i8(d_tmem, da + 2 * kk, db + 2 * kk, p.idesc, (kb | kk) != 0);
                     umma_commit(&sm.empty[s]);
                 }
                 if (ok) umma_commit(&sm.tmem_full[buf]);
@@ -314,20 +442,16 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
         __syncwarp();
     } else {
         // ------------------------------------------------------------ epilogue
-        const int quad = warp & 3;                       // tensor-memory lane group of this warp
-        uint32_t tcount = 0;
-        bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
-            const int m0 = (tile % p.tiles_m) * TC_BM, n0 = (tile / p.tiles_m) * BN;
+        uint32_t tcount = 0, refills = 0;
+        int staged_c0 = -1;
+        for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++tcount) {
+            const int p0 = (tile % p.tiles_p) * TC_BP, c0 = (tile / p.tiles_p) * BN;
             const uint32_t buf = tcount & 1, acc_ph = (tcount >> 1) & 1;
-            ok = mbar_wait(&sm.tmem_full[buf], acc_ph, abort_flag);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * BN;
-            epilogue_rows<OUT_MODE, OUT_BITS>(p, t_row, BN, m0 + quad * 32 + lane, m0, quad, lane, n0);
-            tc_fence_before();
-            mbar_arrive(&sm.tmem_empty[buf]);
+            if (!epilogue_tile<OUT_MODE, OUT_BITS>(p, sm.thr, sm.thr_bar, staged_c0, refills, &sm.tmem_full[buf],
+                                                   acc_ph, tmem_base + buf * BN, BN, p0, c0, warp, lane,
+                                                   abort_flag, (int)tcount))
+                break;
+            if (lane == 0) mbar_arrive(&sm.tmem_empty[buf]);     // one arrival per warp
         }
     }
 
@@ -340,8 +464,8 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
 }
 
 // ---------------------------------------------- kernel B: a CTA pair per 256 x 256 tile
-// Two CTAs of a cluster (two SMs) share one tile: each stages 128 weight rows and
-// 128 of the 256 activation rows, and the leader CTA issues cta_group::2 MMAs
+// Two CTAs of a cluster (two SMs) share one tile: each stages 128 activation rows
+// and 128 of the 256 weight rows, and the leader CTA issues cta_group::2 MMAs
 // (M = 256, N = 256) that read both halves, so each SM pulls 32 KB per 128 depth
 // bytes from L2 instead of 48 KB.  No copy is multicast: each CTA loads only what
 // lands in its own shared memory; its completion bytes are counted on the
@@ -349,13 +473,16 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
 constexpr int T2_STAGES = 6;
 constexpr int T2_BN = 256;
 
+template <int OUT_BITS>
 struct Tc2Smem {
-    alignas(1024) uint8_t w[T2_STAGES][TC_BM * TC_BK];
-    alignas(1024) uint8_t a[T2_STAGES][128 * TC_BK];
+    alignas(1024) uint8_t act[T2_STAGES][TC_BP * TC_BK];
+    alignas(1024) uint8_t wgt[T2_STAGES][128 * TC_BK];
+    alignas(16) int thr[T2_BN * thr_slots(OUT_BITS)];
     alignas(8) uint64_t full[T2_STAGES];
     uint64_t empty[T2_STAGES];
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
+    uint64_t thr_bar[2];
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -406,12 +533,13 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar_cluster_addr) {
 
 template <int OUT_MODE, int OUT_BITS>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
-qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a,
+qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_constant__ CUtensorMap map_wgt,
                  const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
-    Tc2Smem &sm = *reinterpret_cast<Tc2Smem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    using Smem = Tc2Smem<OUT_BITS>;
+    Smem &sm = *reinterpret_cast<Smem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     constexpr uint32_t TMEM_COLS = 2 * T2_BN;
-    constexpr uint32_t PAIR_STAGE_BYTES = 2 * (TC_BM + 128) * TC_BK;   // both CTAs' copies of one stage
+    constexpr uint32_t PAIR_STAGE_BYTES = 2 * (TC_BP + 128) * TC_BK;   // both CTAs' copies of one stage
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
@@ -420,7 +548,10 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < T2_STAGES; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&sm.tmem_full[b], 1); mbar_init(&sm.tmem_empty[b], 8); }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&sm.tmem_full[b], 1); mbar_init(&sm.tmem_empty[b], 2 * EPI_WARPS);
+            mbar_init(&sm.thr_bar[b], EPI_WARPS);
+        }
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -429,7 +560,7 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
     cluster_sync_all();
     tc_fence_after();
     const uint32_t tmem_base = sm.tmem_base;
-    const int num_tiles = p.tiles_m * p.tiles_n;       // tiles of 256 x 256
+    const int num_tiles = p.tiles_p * p.tiles_c;       // tiles of 256 pixels x 256 channels
 
     if (warp == 0) {
         // ---------------------------------------- producer (one per CTA, own halves)
@@ -437,16 +568,16 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
             uint32_t it = 0;
             bool ok = true;
             for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
-                const int m0 = (tile % p.tiles_m) * 256 + (int)rank * 128;
-                const int n0 = (tile / p.tiles_m) * T2_BN + (int)rank * 128;
+                const int p0 = (tile % p.tiles_p) * 256 + (int)rank * 128;
+                const int c0 = (tile / p.tiles_p) * T2_BN + (int)rank * 128;
                 for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
                     const int s = it % T2_STAGES;
                     const uint32_t ph = (it / T2_STAGES) & 1;
                     if (!(ok = mbar_wait(&sm.empty[s], ph ^ 1, abort_flag))) break;
                     if (rank == 0) mbar_arrive_expect_tx(&sm.full[s], PAIR_STAGE_BYTES);
                     const uint32_t leader_full = map_to_cta(smem_u32(&sm.full[s]), 0);
-                    tma_load_2d_pair(sm.w[s], &map_w, leader_full, kb * TC_BK, m0);
-                    tma_load_2d_pair(sm.a[s], &map_a, leader_full, kb * TC_BK, n0);
+                    tma_load_2d_pair(sm.act[s], &map_act, leader_full, kb * TC_BK, p0);
+                    tma_load_2d_pair(sm.wgt[s], &map_wgt, leader_full, kb * TC_BK, c0);
                 }
             }
         }
@@ -466,11 +597,11 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                     const uint32_t ph = (it / T2_STAGES) & 1;
                     if (!(ok = mbar_wait(&sm.full[s], ph, abort_flag))) break;
                     tc_fence_after();
-                    const uint64_t dw = umma_smem_desc(smem_u32(sm.w[s]));
-                    const uint64_t da = umma_smem_desc(smem_u32(sm.a[s]));
+                    const uint64_t da = umma_smem_desc(smem_u32(sm.act[s]));
+                    const uint64_t db = umma_smem_desc(smem_u32(sm.wgt[s]));
 #pragma unroll
                     for (int kk = 0; kk < TC_BK / 32; ++kk)
-                        umma_i8_pair(d_tmem, dw + 2 * kk, da + 2 * kk, p.idesc, (kb | kk) != 0);
+                        umma_i8_pair(d_tmem, da + 2 * kk, db + 2 * kk, p.idesc, (kb | kk) != 0);
                     // free the stage in both CTAs
                     umma_commit_pair(map_to_cta(smem_u32(&sm.empty[s]), 0));
                     umma_commit_pair(map_to_cta(smem_u32(&sm.empty[s]), 1));
@@ -483,21 +614,16 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         }
         __syncwarp();
     } else {
-        // ------------------------------------------- epilogue (each CTA: its 128 rows)
-        const int quad = warp & 3;
-        uint32_t tcount = 0;
-        bool ok = true;
-        for (int tile = pair; ok && tile < num_tiles; tile += num_pairs, ++tcount) {
-            const int m0 = (tile % p.tiles_m) * 256 + (int)rank * 128, n0 = (tile / p.tiles_m) * T2_BN;
+        // ----------------------------- epilogue (each CTA: its 128 pixels, all 256 channels)
+        uint32_t tcount = 0, refills = 0;
+        int staged_c0 = -1;
+        for (int tile = pair; tile < num_tiles; tile += num_pairs, ++tcount) {
+            const int p0 = (tile % p.tiles_p) * 256 + (int)rank * 128, c0 = (tile / p.tiles_p) * T2_BN;
             const uint32_t buf = tcount & 1, acc_ph = (tcount >> 1) & 1;
-            ok = mbar_wait(&sm.tmem_full[buf], acc_ph, abort_flag);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * T2_BN;
-            epilogue_rows<OUT_MODE, OUT_BITS>(p, t_row, T2_BN, m0 + quad * 32 + lane, m0, quad, lane, n0);
-            tc_fence_before();
-            __syncwarp();
+            if (!epilogue_tile<OUT_MODE, OUT_BITS>(p, sm.thr, sm.thr_bar, staged_c0, refills, &sm.tmem_full[buf],
+                                                   acc_ph, tmem_base + buf * T2_BN, T2_BN, p0, c0, warp, lane,
+                                                   abort_flag))
+                break;
             if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&sm.tmem_empty[buf]), 0));
         }
     }
@@ -543,36 +669,36 @@ static bool make_map(CUtensorMap *map, const void *base, int rows, int K, int ld
 }
 
 template <int BN, int STAGES, int OUT_MODE, int OUT_BITS>
-static qnn_status launch_cfg(const CUtensorMap &mw, const CUtensorMap &ma, const TcParams &p, cudaStream_t s) {
+static qnn_status launch_cfg(const CUtensorMap &ma, const CUtensorMap &mw, const TcParams &p, cudaStream_t s) {
     auto kern = qgemm_tc_kernel<BN, STAGES, OUT_MODE, OUT_BITS>;
-    const size_t smem = sizeof(TcSmem<BN, STAGES>) + 1024;
+    const size_t smem = sizeof(TcSmem<BN, STAGES, OUT_BITS>) + 1024;
     static bool attr_done = false;        // per instantiation
     if (!attr_done) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return QNN_ERR_CUDA;
         attr_done = true;
     }
-    const int tiles = p.tiles_m * p.tiles_n;
+    const int tiles = p.tiles_p * p.tiles_c;
     const int grid = tiles < sm_count() ? tiles : sm_count();
-    kern<<<grid, TC_THREADS, smem, s>>>(mw, ma, p);
+    kern<<<grid, TC_THREADS, smem, s>>>(ma, mw, p);
     count_launch();
     return launch_status();
 }
 
 template <int OUT_MODE, int OUT_BITS>
-static qnn_status launch_pair_cfg(const CUtensorMap &mw, const CUtensorMap &ma, const TcParams &p, cudaStream_t s) {
+static qnn_status launch_pair_cfg(const CUtensorMap &ma, const CUtensorMap &mw, const TcParams &p, cudaStream_t s) {
     auto kern = qgemm_tc2_kernel<OUT_MODE, OUT_BITS>;
-    const size_t smem = sizeof(Tc2Smem) + 1024;
+    const size_t smem = sizeof(Tc2Smem<OUT_BITS>) + 1024;
     static bool attr_done = false;
     if (!attr_done) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return QNN_ERR_CUDA;
         attr_done = true;
     }
-    const int tiles = p.tiles_m * p.tiles_n;
+    const int tiles = p.tiles_p * p.tiles_c;
     const int max_pairs = sm_count() / 2;
     const int pairs = tiles < max_pairs ? tiles : max_pairs;
-    kern<<<2 * pairs, TC_THREADS, smem, s>>>(mw, ma, p);
+    kern<<<2 * pairs, TC_THREADS, smem, s>>>(ma, mw, p);
     count_launch();
     return launch_status();
 }
@@ -588,16 +714,16 @@ static qnn_status launch_pair_cfg(const CUtensorMap &mw, const CUtensorMap &ma, 
     return QNN_ERR_UNSUPPORTED;
 
 template <int BN, int STAGES>
-static qnn_status launch_out(int mode, int out_bits, const CUtensorMap &mw, const CUtensorMap &ma,
+static qnn_status launch_out(int mode, int out_bits, const CUtensorMap &ma, const CUtensorMap &mw,
                              const TcParams &p, cudaStream_t s) {
-#define QNN_C1(MODE_, BITS_) launch_cfg<BN, STAGES, MODE_, BITS_>(mw, ma, p, s)
+#define QNN_C1(MODE_, BITS_) launch_cfg<BN, STAGES, MODE_, BITS_>(ma, mw, p, s)
     QNN_TC_DISPATCH(QNN_C1(OUT_RAW, 0), QNN_C1)
 #undef QNN_C1
 }
 
-static qnn_status launch_pair_out(int mode, int out_bits, const CUtensorMap &mw, const CUtensorMap &ma,
+static qnn_status launch_pair_out(int mode, int out_bits, const CUtensorMap &ma, const CUtensorMap &mw,
                                   const TcParams &p, cudaStream_t s) {
-#define QNN_C2(MODE_, BITS_) launch_pair_cfg<MODE_, BITS_>(mw, ma, p, s)
+#define QNN_C2(MODE_, BITS_) launch_pair_cfg<MODE_, BITS_>(ma, mw, p, s)
     QNN_TC_DISPATCH(QNN_C2(OUT_RAW, 0), QNN_C2)
 #undef QNN_C2
 }
@@ -607,13 +733,7 @@ static bool choose_pair_kernel(const qnn_gemm_desc *d, int sms) {
     const char *force = getenv("QNN_TC_KERNEL");
     if (force && force[0] == 's') return false;
     if (force && force[0] == 'p') return true;
-    if (d->N < 256 || d->M <= 128) return false;
-    // estimated time in units of 128x256-tile main loops; a pair tile runs ~0.75 of two of those
-    const long long t1 = (long long)ceil_div(d->M, 128) * ceil_div(d->N, 256);
-    const long long t2 = (long long)ceil_div(d->M, 256) * ceil_div(d->N, 256);
-    const double cost1 = (double)ceil_div((int)t1, sms);
-    const double cost2 = 0.75 * (double)ceil_div((int)t2, sms / 2);
-    return t1 >= sms && cost2 < cost1;
+    return false;
 }
 
 qnn_status gemm_tc_launch(const qnn_gemm_desc *d, const void *W, const void *A, const int32_t *thr,
@@ -630,35 +750,41 @@ qnn_status gemm_tc_launch(const qnn_gemm_desc *d, const void *W, const void *A, 
                         : (d->w_enc == QNN_ENC_SIGNED ? double(1 << (d->w_bits - 1)) : double((1 << d->w_bits) - 1));
     const double amax = d->a_enc == QNN_ENC_BIPOLAR ? 1.0
                         : (d->a_enc == QNN_ENC_SIGNED ? double(1 << (d->a_bits - 1)) : double((1 << d->a_bits) - 1));
-    p.fp_count = (double(d->K) * wmax * amax < 16777216.0) ? 1 : 0;
+    p.fp_count = (double(d->K) * wmax * amax < double(FP_LIMIT)) ? 1 : 0;
     const uint32_t w_s8 = d->w_enc == QNN_ENC_UNSIGNED ? 0u : 1u;
     const uint32_t a_s8 = d->a_enc == QNN_ENC_UNSIGNED ? 0u : 1u;
     const uint32_t idesc_base = (2u << 4)      // accumulator format: s32
-                                | (w_s8 << 7)  // A-operand (weights) format: 0 = u8, 1 = s8
-                                | (a_s8 << 10);   // B-operand (activations) format; both K-major
+                                | (a_s8 << 7)  // MMA A operand = activations: 0 = u8, 1 = s8
+                                | (w_s8 << 10);   // MMA B operand = weights; both K-major
     const int mode = !thr ? OUT_RAW : (d->out_fmt == QNN_FMT_INT8 ? OUT_U8 : OUT_PLANES);
-    CUtensorMap mw, ma;
+    CUtensorMap ma, mw;
 
     if (pair) {
-        if (!make_map(&mw, W, d->M, d->K, ld, TC_BM) || !make_map(&ma, A, d->N, d->K, ld, 128)) return QNN_ERR_CUDA;
-        p.tiles_m = ceil_div(d->M, 256); p.tiles_n = ceil_div(d->N, T2_BN);
+        if (!make_map(&ma, A, d->N, d->K, ld, TC_BP) || !make_map(&mw, W, d->M, d->K, ld, 128)) return QNN_ERR_CUDA;
+        p.tiles_p = ceil_div(d->N, 256); p.tiles_c = ceil_div(d->M, T2_BN);
         p.idesc = idesc_base | ((uint32_t)(T2_BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
-        return launch_pair_out(mode, d->out_bits, mw, ma, p, s);
+        return launch_pair_out(mode, d->out_bits, ma, mw, p, s);
     }
-    // column tile: the widest that still gives every SM a tile
-    const int tiles_m = ceil_div(d->M, TC_BM);
+    // channel tile: the widest that still gives every SM a tile
+    const int tiles_p = ceil_div(d->N, TC_BP);
     int bn = 256;
-    while (bn > 32 && (long long)tiles_m * ceil_div(d->N, bn) < sms) bn >>= 1;
+    while (bn > 32 && (bn / 2 >= round_up(d->M, 32) || (long long)tiles_p * ceil_div(d->M, bn) < sms)) bn >>= 1;
     if (bn == 64) bn = 32;
-    if (!make_map(&mw, W, d->M, d->K, ld, TC_BM) || !make_map(&ma, A, d->N, d->K, ld, bn)) return QNN_ERR_CUDA;
-    p.tiles_m = tiles_m; p.tiles_n = ceil_div(d->N, bn);
-    p.idesc = idesc_base | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+    if (!make_map(&ma, A, d->N, d->K, ld, TC_BP) || !make_map(&mw, W, d->M, d->K, ld, bn)) return QNN_ERR_CUDA;
+    p.tiles_p = tiles_p; p.tiles_c = ceil_div(d->M, bn);
+    p.idesc = idesc_base | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(TC_BP >> 4) << 24);
     switch (bn) {
-        case 256: return launch_out<256, 4>(mode, d->out_bits, mw, ma, p, s);
-        case 128: return launch_out<128, 6>(mode, d->out_bits, mw, ma, p, s);
-        default:  return launch_out<32, 8>(mode, d->out_bits, mw, ma, p, s);
+        case 256: return launch_out<256, 4>(mode, d->out_bits, ma, mw, p, s);
+        case 128: return launch_out<128, 6>(mode, d->out_bits, ma, mw, p, s);
+        default:  return launch_out<32, 8>(mode, d->out_bits, ma, mw, p, s);
     }
 }
+
+#ifdef QNN_TC_TRACE
+extern "C" int qnn_debug_read_trace(long long *host, int n) {
+    return (int)cudaMemcpyFromSymbol(host, g_trace, sizeof(long long) * n);
+}
+#endif
 
 qnn_status device_status_read(int *status) {
     int v = 0;
