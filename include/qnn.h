@@ -169,6 +169,33 @@ qnn_status qnn_qconv(const qnn_conv_desc *d, const void *Wpacked, const void *in
                      const int32_t *thr, void *out,
                      void *workspace, size_t workspace_bytes, void *stream);
 
+/* Largest lowered matrix, in bytes, that qnn_qconv_static accepts. */
+#define QNN_QCONV_STATIC_MAX_BYTES (16u << 20)
+
+/* Convolution for callers that have no device memory to give as workspace and no
+ * means of getting any.  (The paper has no counterpart; this is a deployment aid.)
+ * Typical cases: a layer plug-in inside an inference server that carves up all
+ * device memory at start-up and hands the plug-in nothing but its input and
+ * output tensors; a control loop with a latency bound, where cudaMalloc may not
+ * be called because it can stall on the whole device.  Same computation, arguments, output and error codes as
+ * qnn_qconv, minus the workspace: the lowered matrix lives in an array that is
+ * part of the library image (QNN_QCONV_STATIC_MAX_BYTES of device memory on
+ * every GPU that loads the library, held until the process exits).  The call
+ * allocates and frees nothing, on the device or through any library.
+ *  - Problems whose lowered matrix (qnn_conv_workspace_bytes) is larger than
+ *    QNN_QCONV_STATIC_MAX_BYTES are refused with QNN_ERR_WORKSPACE before
+ *    anything is launched.
+ *  - The first call on each device looks up the array's device address (with
+ *    that device current); make that first call before any stream capture
+ *    begins on the device.
+ *  - All calls on a device share the one array, and it keeps whatever the
+ *    previous call left in it.  Nothing in it has to start at zero: every call
+ *    rewrites, padding included, all of the lowered matrix it reads.  Two calls
+ *    whose kernels can overlap on the GPU (different streams, no dependency)
+ *    race on the array; order them on one stream or with events. */
+qnn_status qnn_qconv_static(const qnn_conv_desc *d, const void *Wpacked, const void *in,
+                            const int32_t *thr, void *out, void *stream);
+
 /* ---- integer max-pool on activation codes (Section 4.2) ------------------- */
 
 typedef struct {

@@ -35,7 +35,7 @@ EXPORTS = (
     "qnn_packed_ld", "qnn_packed_bytes", "qnn_pack", "qnn_gemm_workspace_bytes",
     "qnn_gemm_out_bytes", "qnn_qgemm", "qnn_conv_out_h", "qnn_conv_out_w",
     "qnn_conv_lowered_k", "qnn_conv_lowered_bytes", "qnn_conv_workspace_bytes",
-    "qnn_conv_out_bytes", "qnn_im2col", "qnn_qconv", "qnn_maxpool",
+    "qnn_conv_out_bytes", "qnn_im2col", "qnn_qconv", "qnn_qconv_static", "qnn_maxpool",
     "qnn_validate_thresholds", "qnn_device_status", "qnn_launch_count",
     "qnn_status_string", "qnn_version",
 )
@@ -87,6 +87,8 @@ _lib.qnn_im2col.restype = _ci
 _lib.qnn_im2col.argtypes = [_P(qnn_conv_desc), _vp, _vp, _vp]
 _lib.qnn_qconv.restype = _ci
 _lib.qnn_qconv.argtypes = [_P(qnn_conv_desc), _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.qnn_qconv_static.restype = _ci
+_lib.qnn_qconv_static.argtypes = [_P(qnn_conv_desc), _vp, _vp, _vp, _vp, _vp]
 _lib.qnn_maxpool.restype = _ci
 _lib.qnn_maxpool.argtypes = [_P(qnn_pool_desc), _vp, _vp, _vp]
 _lib.qnn_validate_thresholds.restype = _ci
@@ -198,6 +200,16 @@ def qnn_im2col(d, inp, lowered, stream=None) -> int:
 def qnn_qconv(d, Wpacked, inp, thr, out, workspace, workspace_bytes, stream=None) -> int:
     return _lib.qnn_qconv(ctypes.byref(d), _ptr(Wpacked), _ptr(inp), _ptr(thr), _ptr(out),
                           _ptr(workspace), workspace_bytes, _stream(stream))
+
+
+QNN_QCONV_STATIC_MAX_BYTES = 16 << 20
+
+
+def qnn_qconv_static(d, Wpacked, inp, thr, out, stream=None) -> int:
+    """qnn_qconv without a workspace argument: the lowered matrix goes into a fixed
+    array inside the library, so the call allocates nothing (see include/qnn.h)."""
+    return _lib.qnn_qconv_static(ctypes.byref(d), _ptr(Wpacked), _ptr(inp), _ptr(thr), _ptr(out),
+                                 _stream(stream))
 
 
 def qnn_maxpool(d, inp, out, stream=None) -> int:

@@ -212,6 +212,43 @@ qnn_status qnn_qconv(const qnn_conv_desc *d, const void *Wpacked, const void *in
     return qnn_qgemm(&g, Wpacked, workspace, thr, out, nullptr, 0, stream);
 }
 
+// Lowered-matrix storage of qnn_qconv_static.  In host code this name is only a
+// handle for cudaGetSymbolAddress; the kernels get the address that call returns.
+static __device__ __align__(256) unsigned char g_static_lowered[QNN_QCONV_STATIC_MAX_BYTES];
+
+// Device address of g_static_lowered on the current device, looked up once per device.
+static qnn_status static_lowered_ptr(void **ptr) {
+    static void *cached[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return QNN_ERR_CUDA;
+    if (!cached[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_lowered) != cudaSuccess || !p) return QNN_ERR_CUDA;
+        cached[dev] = p;
+    }
+    *ptr = cached[dev];
+    return QNN_OK;
+}
+
+qnn_status qnn_qconv_static(const qnn_conv_desc *d, const void *Wpacked, const void *in, const int32_t *thr,
+                            void *out, void *stream) {
+    qnn_status st = check_conv_desc(d);
+    if (st != QNN_OK) return st;
+    qnn_gemm_desc g;
+    conv_to_gemm(d, &g);
+    st = check_gemm_desc(&g, thr != nullptr, nullptr);
+    if (st != QNN_OK) return st;
+    if (qnn_conv_workspace_bytes(d) > (size_t)QNN_QCONV_STATIC_MAX_BYTES) return QNN_ERR_WORKSPACE;
+    if (!Wpacked || !in || !out) return QNN_ERR_INVALID_ARG;
+    if (!aligned16(Wpacked) || !aligned16(in) || !aligned16(out)) return QNN_ERR_ALIGNMENT;
+    void *lowered = nullptr;
+    st = static_lowered_ptr(&lowered);
+    if (st != QNN_OK) return st;
+    st = im2col_launch(d, in, lowered, (cudaStream_t)stream);
+    if (st != QNN_OK) return st;
+    return qnn_qgemm(&g, Wpacked, lowered, thr, out, nullptr, 0, stream);
+}
+
 qnn_status qnn_maxpool(const qnn_pool_desc *d, const void *in, void *out, void *stream) {
     if (!d || !in || !out) return QNN_ERR_INVALID_ARG;
     if (d->B <= 0 || d->H <= 0 || d->W <= 0 || d->C <= 0 || d->k <= 0 || d->stride <= 0)
