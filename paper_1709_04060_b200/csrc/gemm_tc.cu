@@ -15,16 +15,23 @@
 // 16-byte stores, and the 32 bits of one plane are one word of the
 // channel-interleaved layout of Section 3.2.
 //
-// Kernel structure (persistent, one CTA per SM, 320 threads):
+// Kernel structure (persistent, one CTA per SM, 352 threads):
 //   warp 0     TMA producer: 128-byte-swizzled K-major tiles of the activations
 //              (128 rows) and weights (BN rows) into a shared-memory ring
 //   warp 1     allocates tensor memory; one lane issues the MMAs
 //              (M = 128, N = BN, K = 32 per instruction) and commits to mbarriers
-//   warps 2-9  epilogue: warp e reads lanes 32*(e%4).. and the column half e/4;
-//              thresholds of the tile's channels are staged in shared memory.
+//   warps 2-9  epilogue: warp e reads lanes 32*(e%4).. and the column half e/4
+//   warp 10    threshold stager: loads the thresholds of the next work unit's
+//              channels, sorts each channel's set (the count does not depend on
+//              their order) and writes them to one of two shared-memory buffers
 // Two accumulator buffers in tensor memory let the epilogue of tile t overlap the
 // main loop of tile t+1.  Every wait is bounded; on expiry the CTA records
 // QNN_ERR_DEVICE_TIMEOUT in the device status word, drains and exits.
+//
+// Work units: 128 x BN tiles dealt round-robin to the CTAs.  When the last round
+// would fill only part of the GPU, its tiles are cut along the channels into
+// 2, 4 or 8 narrower units (MMA N = BN/2 ..), so that the round costs a fraction of
+// a full tile instead of a whole one.
 #include <cuda.h>
 #include <stdlib.h>
 
@@ -131,7 +138,29 @@ struct TcParams {
     int ld_out;            // INT8 output row pitch
     int fp_count;          // 1: |acc| < 2^22, thresholds are counted on the FP32 pipe
     uint32_t idesc;
+    // work units: [0, full_units) are whole tiles, then every remaining tile is cut
+    // into `split` units of bn_sub channels each
+    int units, full_units, split, bn_sub;
+    uint32_t idesc_sub;
 };
+
+struct TcUnit { int p0, c0, bn; bool sub; };
+
+__device__ __forceinline__ TcUnit tc_unit(const TcParams &p, int u, int bn_full) {
+    TcUnit r;
+    int tile = u, part = 0;
+    r.sub = u >= p.full_units;
+    r.bn = bn_full;
+    if (r.sub) {
+        const int j = u - p.full_units;
+        tile = p.full_units + j / p.split;
+        part = j - (j / p.split) * p.split;
+        r.bn = p.bn_sub;
+    }
+    r.p0 = (tile % p.tiles_p) * TC_BP;
+    r.c0 = (tile / p.tiles_p) * bn_full + part * r.bn;
+    return r;
+}
 
 enum { OUT_RAW = 0, OUT_U8 = 1, OUT_PLANES = 2 };
 
@@ -146,7 +175,8 @@ enum { OUT_RAW = 0, OUT_U8 = 1, OUT_PLANES = 2 };
 // accumulated in one float on top of 1.5*2^23 (the second scaled by 256), so the
 // two codes are the low two bytes of the sum's bit pattern.
 constexpr int EPI_WARPS = 8;
-constexpr int TC_THREADS = 64 + 32 * EPI_WARPS;
+constexpr int STAGER_WARP = 2 + EPI_WARPS;
+constexpr int TC_THREADS = 64 + 32 * EPI_WARPS + 32;
 constexpr float FP_MAGIC = 12582912.0f;        // 1.5 * 2^23, bit pattern 0x4B400000
 constexpr int FP_MAGIC_BITS = 0x4B400000;
 constexpr int FP_LIMIT = 1 << 22;
@@ -183,21 +213,42 @@ __device__ __forceinline__ uint32_t nibble_of_plane(uint32_t x, int b) {
     return (((x >> b) & 0x01010101u) * 0x01020408u) >> 24;
 }
 
-// Stage the thresholds of channels [c0, c0 + bn) in shared memory: float form for the
-// FP count, raw int32 otherwise; slots past the row's thresholds and channels past M
-// hold a value no accumulator reaches.
+// Stage the thresholds of channels [c0, c0 + bn) in shared memory (one warp, a lane per
+// channel).  Slots past the row's thresholds and channels past M hold a value no
+// accumulator reaches.  Sets of 7 or 15 thresholds are sorted so that the epilogue can
+// count by bisection (raw int32); sets of 1 or 3 are counted linearly, in float form
+// when the FP count applies.
 template <int OUT_BITS>
-__device__ __forceinline__ void stage_thresholds(const TcParams &p, int *thr_s, int c0, int bn, int etid) {
+__device__ __forceinline__ void stage_thresholds(const TcParams &p, int *thr_s, int c0, int bn, int lane) {
     constexpr int N_THR = (1 << OUT_BITS) - 1, NT = thr_slots(OUT_BITS);
-    for (int idx = etid; idx < bn * NT; idx += 32 * EPI_WARPS) {
-        const int c = idx / NT, q = idx - c * NT, m = c0 + c;
-        int t = 0x7fffffff;
-        if (q < N_THR && m < p.M) t = p.thr[(size_t)m * N_THR + q];
-        if (p.fp_count) {
-            const int tc = t <= -FP_LIMIT ? -FP_LIMIT + 1 : (t > FP_LIMIT ? FP_LIMIT : t);
-            t = FP_MAGIC_BITS + (tc - 1);
+    for (int c = lane; c < bn; c += 32) {
+        const int m = c0 + c;
+        int t[NT];
+#pragma unroll
+        for (int q = 0; q < NT; ++q) t[q] = 0x7fffffff;
+        if (m < p.M) {
+#pragma unroll
+            for (int q = 0; q < N_THR; ++q) t[q] = __ldg(p.thr + (size_t)m * N_THR + q);
         }
-        thr_s[idx] = t;
+        if (OUT_BITS >= 3) {
+            // odd-even transposition sort; the pads are the largest value and stay last
+#pragma unroll
+            for (int r = 0; r < NT; ++r)
+#pragma unroll
+                for (int i = r & 1; i + 1 < NT; i += 2) {
+                    const int lo = min(t[i], t[i + 1]), hi = max(t[i], t[i + 1]);
+                    t[i] = lo; t[i + 1] = hi;
+                }
+        } else if (p.fp_count) {
+#pragma unroll
+            for (int q = 0; q < NT; ++q) {
+                const int tc = t[q] <= -FP_LIMIT ? -FP_LIMIT + 1 : (t[q] > FP_LIMIT ? FP_LIMIT : t[q]);
+                t[q] = FP_MAGIC_BITS + (tc - 1);
+            }
+        }
+#pragma unroll
+        for (int v = 0; v < NT / 4; ++v)
+            reinterpret_cast<int4 *>(thr_s + c * NT)[v] = make_int4(t[4 * v], t[4 * v + 1], t[4 * v + 2], t[4 * v + 3]);
     }
 }
 
@@ -221,7 +272,24 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams &p, const int *thr
         return;
     }
     uint32_t packed[8];                          // four codes per word, one byte each
-    if (p.fp_count) {
+    if (OUT_BITS >= 3) {
+        // bisection over the channel's sorted thresholds: the row of NT words sits in NT
+        // distinct banks, so lanes that look at different slots do not conflict
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            uint32_t w = 0;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int j = 4 * k + e, x = acc[j];
+                const int *row = thr_c + j * NT;
+                int c = (x >= row[NT / 2 - 1]) ? NT / 2 : 0;
+#pragma unroll
+                for (int step = NT / 4; step >= 1; step >>= 1) c += (x >= row[c + step - 1]) ? step : 0;
+                w |= (uint32_t)c << (8 * e);
+            }
+            packed[k] = w;
+        }
+    } else if (p.fp_count) {
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             uint32_t pr[2];
@@ -303,38 +371,44 @@ __device__ __forceinline__ void epilogue_cols(const TcParams &p, const int *thr_
     }
 }
 
-// Epilogue warps meet on an mbarrier (bounded wait) instead of a named barrier.
-__device__ __forceinline__ bool epi_sync(uint64_t *bar, uint32_t parity, int lane, volatile int *abort_flag) {
-    __syncwarp();
+// One lane polls the barrier, the warp follows.
+__device__ __forceinline__ bool warp_wait(uint64_t *bar, uint32_t parity, int lane, volatile int *abort_flag) {
     bool ok = true;
-    if (lane == 0) {
-        mbar_arrive(bar);
-        ok = mbar_wait(bar, parity, abort_flag);
-    }
+    if (lane == 0) ok = mbar_wait(bar, parity, abort_flag);
     return __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
 }
 
-// Per-tile epilogue shared by both kernels.  Returns false if a wait ran out.
+// Threshold stager (one warp): unit i of this CTA uses threshold buffer i & 1.
+// `next_unit(i, c0, bn)` yields the channel range of the CTA's i-th unit, false past the end.
+template <int OUT_BITS, int BN, typename NextUnit>
+__device__ __forceinline__ void stager_loop(const TcParams &p, int *thr_s, uint64_t *thr_full, uint64_t *thr_empty,
+                                            int lane, volatile int *abort_flag, NextUnit next_unit) {
+    constexpr int NT = thr_slots(OUT_BITS);
+    int c0, bn;
+    for (uint32_t i = 0; next_unit(i, c0, bn); ++i) {
+        const uint32_t b = i & 1, ph = (i >> 1) & 1;
+        if (!warp_wait(&thr_empty[b], ph ^ 1, lane, abort_flag)) return;
+        stage_thresholds<OUT_BITS>(p, thr_s + b * BN * NT, c0, bn, lane);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&thr_full[b]);
+    }
+}
+
+// Per-unit epilogue shared by both kernels: waits for the unit's thresholds and for its
+// accumulators, processes this warp's part, then releases the threshold buffer (the
+// caller releases the accumulators).  Returns false if a wait ran out.
 template <int OUT_MODE, int OUT_BITS>
-__device__ __forceinline__ bool epilogue_tile(const TcParams &p, int *thr_s, uint64_t *thr_bar, int &staged_c0,
-                                              uint32_t &refills, uint64_t *tmem_full, uint32_t full_parity,
+__device__ __forceinline__ bool epilogue_tile(const TcParams &p, const int *thr_s, uint64_t *thr_full,
+                                              uint64_t *thr_empty, uint32_t thr_parity,
+                                              uint64_t *tmem_full, uint32_t full_parity,
                                               uint32_t t_acc, int bn, int p0, int c0, int warp, int lane,
                                               volatile int *abort_flag, int full_parity_dbg = 0) {
     const int quad = warp & 3, half = (warp - 2) >> 2;
     const bool tr = warp == 2 && lane == 0;
     if (tr) QNN_TRACE(0, full_parity_dbg);
-    if (OUT_MODE != OUT_RAW && staged_c0 != c0) {
-        // everyone is done with the old thresholds -> refill -> everyone sees the new ones
-        if (!epi_sync(&thr_bar[0], refills & 1, lane, abort_flag)) return false;
-        stage_thresholds<OUT_BITS>(p, thr_s, c0, bn, (warp - 2) * 32 + lane);
-        if (!epi_sync(&thr_bar[1], refills & 1, lane, abort_flag)) return false;
-        ++refills;
-        staged_c0 = c0;
-    }
-    bool ok = true;
+    if (OUT_MODE != OUT_RAW && !warp_wait(thr_full, thr_parity, lane, abort_flag)) return false;
     if (tr) QNN_TRACE(1, full_parity_dbg);
-    if (lane == 0) ok = mbar_wait(tmem_full, full_parity, abort_flag);    // one lane polls
-    if (__shfl_sync(0xffffffffu, (int)ok, 0) == 0) return false;
+    if (!warp_wait(tmem_full, full_parity, lane, abort_flag)) return false;
     if (tr) QNN_TRACE(2, full_parity_dbg);
     tc_fence_after();
     const int hcols = bn >= 64 ? bn / 2 : bn;
@@ -343,6 +417,7 @@ __device__ __forceinline__ bool epilogue_tile(const TcParams &p, int *thr_s, uin
                                       p0 + quad * 32 + lane, c0);
     tc_fence_before();
     __syncwarp();
+    if (OUT_MODE != OUT_RAW && lane == 0) mbar_arrive(thr_empty);
     if (tr) QNN_TRACE(3, full_parity_dbg);
     return true;
 }
@@ -352,12 +427,13 @@ template <int BN, int STAGES, int OUT_BITS>
 struct TcSmem {
     alignas(1024) uint8_t act[STAGES][TC_BP * TC_BK];
     alignas(1024) uint8_t wgt[STAGES][BN * TC_BK];
-    alignas(16) int thr[BN * thr_slots(OUT_BITS)];
+    alignas(16) int thr[2][BN * thr_slots(OUT_BITS)];
     alignas(8) uint64_t full[STAGES];
     uint64_t empty[STAGES];
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
-    uint64_t thr_bar[2];
+    uint64_t thr_full[2];
+    uint64_t thr_empty[2];
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -365,12 +441,11 @@ struct TcSmem {
 template <int BN, int STAGES, int OUT_MODE, int OUT_BITS>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_constant__ CUtensorMap map_wgt,
-                const TcParams p) {
+                const __grid_constant__ CUtensorMap map_wgt_sub, const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
     using Smem = TcSmem<BN, STAGES, OUT_BITS>;
     Smem &sm = *reinterpret_cast<Smem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     constexpr uint32_t TMEM_COLS = (2 * BN < 32) ? 32 : 2 * BN;
-    constexpr uint32_t STAGE_BYTES = (TC_BP + BN) * TC_BK;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int *abort_flag = &sm.abort_flag;
@@ -379,7 +454,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
         for (int s = 0; s < STAGES; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&sm.tmem_full[b], 1); mbar_init(&sm.tmem_empty[b], EPI_WARPS);
-            mbar_init(&sm.thr_bar[b], EPI_WARPS);
+            mbar_init(&sm.thr_full[b], 1); mbar_init(&sm.thr_empty[b], EPI_WARPS);
         }
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -389,22 +464,23 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = sm.tmem_base;
-    const int num_tiles = p.tiles_p * p.tiles_c;
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-                const int p0 = (tile % p.tiles_p) * TC_BP, c0 = (tile / p.tiles_p) * BN;
+            for (int u = blockIdx.x; ok && u < p.units; u += gridDim.x) {
+                const TcUnit un = tc_unit(p, u, BN);
+                const CUtensorMap *mw = un.sub ? &map_wgt_sub : &map_wgt;
+                const uint32_t stage_bytes = (uint32_t)(TC_BP + un.bn) * TC_BK;
                 for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1;
                     if (!(ok = mbar_wait(&sm.empty[s], ph ^ 1, abort_flag))) break;
-                    mbar_arrive_expect_tx(&sm.full[s], STAGE_BYTES);
-                    tma_load_2d(sm.act[s], &map_act, &sm.full[s], kb * TC_BK, p0);
-                    tma_load_2d(sm.wgt[s], &map_wgt, &sm.full[s], kb * TC_BK, c0);
+                    mbar_arrive_expect_tx(&sm.full[s], stage_bytes);
+                    tma_load_2d(sm.act[s], &map_act, &sm.full[s], kb * TC_BK, un.p0);
+                    tma_load_2d(sm.wgt[s], mw, &sm.full[s], kb * TC_BK, un.c0);
                 }
             }
             if (!ok) {
@@ -419,8 +495,9 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
         if (lane == 0) {
             uint32_t it = 0, tcount = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tcount) {
+            for (int u = blockIdx.x; ok && u < p.units; u += gridDim.x, ++tcount) {
                 const uint32_t buf = tcount & 1, acc_ph = (tcount >> 1) & 1;
+                const uint32_t idesc = u >= p.full_units ? p.idesc_sub : p.idesc;
                 if (!(ok = mbar_wait(&sm.tmem_empty[buf], acc_ph ^ 1, abort_flag))) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
@@ -433,23 +510,33 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
                     const uint64_t db = umma_smem_desc(smem_u32(sm.wgt[s]));
 #pragma unroll
                     for (int kk = 0; kk < TC_BK / 32; ++kk)   // 32 depth bytes per MMA: +2 in 16-byte units
-                        umma_i8(d_tmem, da + 2 * kk, db + 2 * kk, p.idesc, (kb | kk) != 0);
+                        umma_i8(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (kb | kk) != 0);
                     umma_commit(&sm.empty[s]);
                 }
                 if (ok) umma_commit(&sm.tmem_full[buf]);
             }
         }
         __syncwarp();
+    } else if (warp == STAGER_WARP) {
+        // ---------------------------------------------------- threshold stager
+        if (OUT_MODE != OUT_RAW)
+            stager_loop<OUT_BITS, BN>(p, &sm.thr[0][0], sm.thr_full, sm.thr_empty, lane, abort_flag,
+                                      [&](uint32_t i, int &c0, int &bn) {
+                                          const long long u = blockIdx.x + (long long)i * gridDim.x;
+                                          if (u >= p.units) return false;
+                                          const TcUnit un = tc_unit(p, (int)u, BN);
+                                          c0 = un.c0; bn = un.bn;
+                                          return true;
+                                      });
     } else {
         // ------------------------------------------------------------ epilogue
-        uint32_t tcount = 0, refills = 0;
-        int staged_c0 = -1;
-        for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++tcount) {
-            const int p0 = (tile % p.tiles_p) * TC_BP, c0 = (tile / p.tiles_p) * BN;
+        uint32_t tcount = 0;
+        for (int u = blockIdx.x; u < p.units; u += gridDim.x, ++tcount) {
+            const TcUnit un = tc_unit(p, u, BN);
             const uint32_t buf = tcount & 1, acc_ph = (tcount >> 1) & 1;
-            if (!epilogue_tile<OUT_MODE, OUT_BITS>(p, sm.thr, sm.thr_bar, staged_c0, refills, &sm.tmem_full[buf],
-                                                   acc_ph, tmem_base + buf * BN, BN, p0, c0, warp, lane,
-                                                   abort_flag, (int)tcount))
+            if (!epilogue_tile<OUT_MODE, OUT_BITS>(p, sm.thr[buf], &sm.thr_full[buf], &sm.thr_empty[buf], acc_ph,
+                                                   &sm.tmem_full[buf], acc_ph, tmem_base + buf * BN, un.bn,
+                                                   un.p0, un.c0, warp, lane, abort_flag, (int)tcount))
                 break;
             if (lane == 0) mbar_arrive(&sm.tmem_empty[buf]);     // one arrival per warp
         }
@@ -477,12 +564,13 @@ template <int OUT_BITS>
 struct Tc2Smem {
     alignas(1024) uint8_t act[T2_STAGES][TC_BP * TC_BK];
     alignas(1024) uint8_t wgt[T2_STAGES][128 * TC_BK];
-    alignas(16) int thr[T2_BN * thr_slots(OUT_BITS)];
+    alignas(16) int thr[2][T2_BN * thr_slots(OUT_BITS)];
     alignas(8) uint64_t full[T2_STAGES];
     uint64_t empty[T2_STAGES];
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
-    uint64_t thr_bar[2];
+    uint64_t thr_full[2];
+    uint64_t thr_empty[2];
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -550,7 +638,7 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_const
         for (int s = 0; s < T2_STAGES; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&sm.tmem_full[b], 1); mbar_init(&sm.tmem_empty[b], 2 * EPI_WARPS);
-            mbar_init(&sm.thr_bar[b], EPI_WARPS);
+            mbar_init(&sm.thr_full[b], 1); mbar_init(&sm.thr_empty[b], EPI_WARPS);
         }
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -613,16 +701,25 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_const
             }
         }
         __syncwarp();
+    } else if (warp == STAGER_WARP) {
+        // ------------------------------------ threshold stager (all 256 channels of the tile)
+        if (OUT_MODE != OUT_RAW)
+            stager_loop<OUT_BITS, T2_BN>(p, &sm.thr[0][0], sm.thr_full, sm.thr_empty, lane, abort_flag,
+                                         [&](uint32_t i, int &c0, int &bn) {
+                                             const long long tile = pair + (long long)i * num_pairs;
+                                             if (tile >= num_tiles) return false;
+                                             c0 = (int)(tile / p.tiles_p) * T2_BN; bn = T2_BN;
+                                             return true;
+                                         });
     } else {
         // ----------------------------- epilogue (each CTA: its 128 pixels, all 256 channels)
-        uint32_t tcount = 0, refills = 0;
-        int staged_c0 = -1;
+        uint32_t tcount = 0;
         for (int tile = pair; tile < num_tiles; tile += num_pairs, ++tcount) {
             const int p0 = (tile % p.tiles_p) * 256 + (int)rank * 128, c0 = (tile / p.tiles_p) * T2_BN;
             const uint32_t buf = tcount & 1, acc_ph = (tcount >> 1) & 1;
-            if (!epilogue_tile<OUT_MODE, OUT_BITS>(p, sm.thr, sm.thr_bar, staged_c0, refills, &sm.tmem_full[buf],
-                                                   acc_ph, tmem_base + buf * T2_BN, T2_BN, p0, c0, warp, lane,
-                                                   abort_flag))
+            if (!epilogue_tile<OUT_MODE, OUT_BITS>(p, sm.thr[buf], &sm.thr_full[buf], &sm.thr_empty[buf], acc_ph,
+                                                   &sm.tmem_full[buf], acc_ph, tmem_base + buf * T2_BN, T2_BN,
+                                                   p0, c0, warp, lane, abort_flag))
                 break;
             if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&sm.tmem_empty[buf]), 0));
         }
@@ -669,7 +766,8 @@ static bool make_map(CUtensorMap *map, const void *base, int rows, int K, int ld
 }
 
 template <int BN, int STAGES, int OUT_MODE, int OUT_BITS>
-static qnn_status launch_cfg(const CUtensorMap &ma, const CUtensorMap &mw, const TcParams &p, cudaStream_t s) {
+static qnn_status launch_cfg(const CUtensorMap &ma, const CUtensorMap &mw, const CUtensorMap &mws,
+                             const TcParams &p, cudaStream_t s) {
     auto kern = qgemm_tc_kernel<BN, STAGES, OUT_MODE, OUT_BITS>;
     const size_t smem = sizeof(TcSmem<BN, STAGES, OUT_BITS>) + 1024;
     static bool attr_done = false;        // per instantiation
@@ -678,9 +776,8 @@ static qnn_status launch_cfg(const CUtensorMap &ma, const CUtensorMap &mw, const
             return QNN_ERR_CUDA;
         attr_done = true;
     }
-    const int tiles = p.tiles_p * p.tiles_c;
-    const int grid = tiles < sm_count() ? tiles : sm_count();
-    kern<<<grid, TC_THREADS, smem, s>>>(ma, mw, p);
+    const int grid = p.units < sm_count() ? p.units : sm_count();
+    kern<<<grid, TC_THREADS, smem, s>>>(ma, mw, mws, p);
     count_launch();
     return launch_status();
 }
@@ -715,8 +812,8 @@ static qnn_status launch_pair_cfg(const CUtensorMap &ma, const CUtensorMap &mw, 
 
 template <int BN, int STAGES>
 static qnn_status launch_out(int mode, int out_bits, const CUtensorMap &ma, const CUtensorMap &mw,
-                             const TcParams &p, cudaStream_t s) {
-#define QNN_C1(MODE_, BITS_) launch_cfg<BN, STAGES, MODE_, BITS_>(ma, mw, p, s)
+                             const CUtensorMap &mws, const TcParams &p, cudaStream_t s) {
+#define QNN_C1(MODE_, BITS_) launch_cfg<BN, STAGES, MODE_, BITS_>(ma, mw, mws, p, s)
     QNN_TC_DISPATCH(QNN_C1(OUT_RAW, 0), QNN_C1)
 #undef QNN_C1
 }
@@ -762,6 +859,7 @@ qnn_status gemm_tc_launch(const qnn_gemm_desc *d, const void *W, const void *A, 
     if (pair) {
         if (!make_map(&ma, A, d->N, d->K, ld, TC_BP) || !make_map(&mw, W, d->M, d->K, ld, 128)) return QNN_ERR_CUDA;
         p.tiles_p = ceil_div(d->N, 256); p.tiles_c = ceil_div(d->M, T2_BN);
+        p.units = p.full_units = p.tiles_p * p.tiles_c; p.split = 1; p.bn_sub = T2_BN; p.idesc_sub = 0;
         p.idesc = idesc_base | ((uint32_t)(T2_BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
         return launch_pair_out(mode, d->out_bits, ma, mw, p, s);
     }
@@ -770,13 +868,29 @@ qnn_status gemm_tc_launch(const qnn_gemm_desc *d, const void *W, const void *A, 
     int bn = 256;
     while (bn > 32 && (bn / 2 >= round_up(d->M, 32) || (long long)tiles_p * ceil_div(d->M, bn) < sms)) bn >>= 1;
     if (bn == 64) bn = 32;
-    if (!make_map(&ma, A, d->N, d->K, ld, TC_BP) || !make_map(&mw, W, d->M, d->K, ld, bn)) return QNN_ERR_CUDA;
     p.tiles_p = tiles_p; p.tiles_c = ceil_div(d->M, bn);
+    // Work units: when the last round of tiles would occupy at most half of the SMs, cut
+    // each of its tiles along the channels so that the round costs 1/split of a tile.
+    const long long tiles = (long long)p.tiles_p * p.tiles_c;
+    if (tiles > 0x3fffffff) return QNN_ERR_UNSUPPORTED;
+    const int grid = tiles < sms ? (int)tiles : sms;
+    const int rem = (int)(tiles % grid);
+    int split = 1;
+    if (rem > 0)
+        while (2 * split * rem <= grid && bn / (2 * split) >= 32) split *= 2;
+    p.split = split; p.bn_sub = bn / split;
+    p.full_units = split > 1 ? (int)tiles - rem : (int)tiles;
+    p.units = p.full_units + (split > 1 ? rem * split : 0);
     p.idesc = idesc_base | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(TC_BP >> 4) << 24);
+    p.idesc_sub = idesc_base | ((uint32_t)(p.bn_sub >> 3) << 17) | ((uint32_t)(TC_BP >> 4) << 24);
+    CUtensorMap mws;
+    if (!make_map(&ma, A, d->N, d->K, ld, TC_BP) || !make_map(&mw, W, d->M, d->K, ld, bn) ||
+        !make_map(&mws, W, d->M, d->K, ld, p.bn_sub))
+        return QNN_ERR_CUDA;
     switch (bn) {
-        case 256: return launch_out<256, 4>(mode, d->out_bits, ma, mw, p, s);
-        case 128: return launch_out<128, 6>(mode, d->out_bits, ma, mw, p, s);
-        default:  return launch_out<32, 8>(mode, d->out_bits, ma, mw, p, s);
+        case 256: return launch_out<256, 4>(mode, d->out_bits, ma, mw, mws, p, s);
+        case 128: return launch_out<128, 6>(mode, d->out_bits, ma, mw, mws, p, s);
+        default:  return launch_out<32, 8>(mode, d->out_bits, ma, mw, mws, p, s);
     }
 }
 

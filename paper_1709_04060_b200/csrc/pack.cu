@@ -58,6 +58,33 @@ __global__ void pack_planes_kernel(const uint8_t *__restrict__ logical, uint32_t
     }
 }
 
+// Per-byte conversion of four logical bytes to their 8-bit containers.
+__device__ __forceinline__ uint32_t container4(uint32_t x, int bits, int enc) {
+    if (enc == QNN_ENC_BIPOLAR) {
+        const uint32_t gt = __vcmpgts4(x, 0u);                  // 0xFF where the byte is > 0
+        return (gt & 0x01010101u) | ~gt;                        // +1 : -1
+    }
+    if (bits == 8) return x;
+    const uint32_t low = x & (0x01010101u * ((1u << bits) - 1u));
+    if (enc == QNN_ENC_UNSIGNED) return low;
+    // sign extension inside every byte: the sign bit, moved up one place, times
+    // 2^(8-bits) - 1 fills bits [bits, 8) and cannot carry into the next byte
+    const uint32_t sign = low & (0x01010101u << (bits - 1));
+    return low | ((sign << 1) * ((1u << (8 - bits)) - 1u));
+}
+
+// K a multiple of 16 (no padding): one thread per 16 bytes, 16-byte loads and stores.
+__global__ void __launch_bounds__(256) pack_int8_vec_kernel(const uint4 *__restrict__ logical,
+                                                            uint4 *__restrict__ packed, long long n16,
+                                                            int bits, int enc) {
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n16;
+         i += (long long)gridDim.x * blockDim.x) {
+        const uint4 v = logical[i];
+        packed[i] = make_uint4(container4(v.x, bits, enc), container4(v.y, bits, enc),
+                               container4(v.z, bits, enc), container4(v.w, bits, enc));
+    }
+}
+
 // One thread per 16 output bytes of the [rows][ld] container matrix.
 __global__ void pack_int8_kernel(const uint8_t *__restrict__ logical, uint8_t *__restrict__ packed,
                                  int rows, int K, int ld, int bits, int enc) {
@@ -109,6 +136,14 @@ qnn_status pack_launch(const qnn_pack_desc *d, const void *logical, void *packed
     } else {
         const int ld = round_up(d->K, 16);
         const long long total = (long long)d->rows * (ld / 16);
+        if (d->K % 16 == 0) {
+            const long long want = (total + threads - 1) / threads;
+            const long long cap = (long long)sm_count() * 16;
+            pack_int8_vec_kernel<<<(unsigned)(want < cap ? want : cap), threads, 0, s>>>(
+                (const uint4 *)logical, (uint4 *)packed, total, d->bits, d->enc);
+            count_launch();
+            return launch_status();
+        }
         const unsigned blocks = (unsigned)((total + threads - 1) / threads);
         pack_int8_kernel<<<blocks, threads, 0, s>>>((const uint8_t *)logical, (uint8_t *)packed,
                                                     d->rows, d->K, ld, d->bits, d->enc);

@@ -158,6 +158,20 @@ def test_both_tensor_core_kernels(qb, force_tc_kernel, which, M, N, K, w, a):
     run_case(qb, case, INT8, INT8, raw=True)
 
 
+@pytest.mark.parametrize("M,N,K,w,a", [
+    (250, 19195, 256, 1, 2),     # 150 tiles on 148 SMs: the last 2 are cut into 8 units of 32 channels
+    (512, 10240, 160, 2, 4),     # 160 tiles: the last 12 are cut into 4 units of 64 channels
+    (768, 8440, 192, 4, 3),      # 198 tiles: the last 50 are cut into 2 units of 128 channels
+])
+def test_partial_last_round_is_cut_into_narrow_units(qb, M, N, K, w, a):
+    """Tile counts just above a multiple of the SM count: the tiles of the last round are
+    split along the channels (narrower MMAs, second weight tensor map); every output checked."""
+    case = synth.gemm_case(1200 + M, M, N, K, w, a)
+    run_case(qb, case, INT8, INT8)
+    run_case(qb, case, INT8, BITPLANES)
+    run_case(qb, case, INT8, INT8, raw=True)
+
+
 @pytest.mark.parametrize("which", ["single", "pair"])
 def test_integer_count_path_for_large_accumulators(qb, force_tc_kernel, which):
     """8-bit x 8-bit with K large enough that |acc| can exceed 2^24: the epilogue must
