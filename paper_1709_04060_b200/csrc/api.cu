@@ -149,6 +149,8 @@ qnn_status qnn_qgemm(const qnn_gemm_desc *d, const void *W, const void *A, const
     if (!aligned16(W) || !aligned16(A) || !aligned16(out) || (thr && (reinterpret_cast<uintptr_t>(thr) & 3u)))
         return QNN_ERR_ALIGNMENT;
     if (path == QNN_PATH_TCGEN05_I8) return gemm_tc_launch(d, W, A, thr, out, (cudaStream_t)stream);
+    // a handful of columns: stream the weight planes once, one warp per row
+    if (gemv_planes_fits(d)) return gemv_planes_launch(d, W, A, thr, out, (cudaStream_t)stream);
     return gemm_bitserial_launch(d, W, A, thr, out, (cudaStream_t)stream);
 }
 

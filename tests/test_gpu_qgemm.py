@@ -210,3 +210,46 @@ def test_full_size_4096_sampled(qb, w, a):
     assert np.array_equal(codes[:, 777].astype(np.int64), full_row)
     full_col = orc.qgemm(case.W, case.At[1234:1235], case.thr)[:, 0]
     assert np.array_equal(codes[1234, :].astype(np.int64), full_col)
+
+
+@pytest.mark.parametrize("fmt", [BITPLANES, INT8])
+@pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("N", [1, 4, 16])
+def test_config5_skinny_fc(qb, fmt, bits, N):
+    """Large fully connected layer at small batch (M = K = 8192, N in {1, 4, 16}), W2A2 and
+    W4A4, signed weights: every output against the oracle, both operand formats."""
+    case = synth.gemm_case(5000 + 10 * bits + N, 8192, N, 8192, bits, bits)
+    run_case(qb, case, fmt, INT8)
+    run_case(qb, case, fmt, BITPLANES)
+    run_case(qb, case, fmt, INT8, raw=True)
+
+
+@pytest.mark.parametrize("w_enc,a_enc,w,a", [(2, 0, 1, 2), (1, 2, 3, 1), (2, 2, 1, 1), (0, 1, 4, 3)])
+def test_skinny_bit_serial_encodings(qb, w_enc, a_enc, w, a):
+    """The few-column bit-serial kernel with bipolar / signed / unsigned operands, depths that
+    are and are not a multiple of 128 (vector and scalar loads), ragged M."""
+    for K, M, N in ((9216, 333, 3), (1000, 70, 16), (4096, 4096, 1)):
+        case = synth.gemm_case(5100 + K + w, M, N, K, w, a, w_enc, a_enc, out_bits=2)
+        run_case(qb, case, BITPLANES, INT8, check_pack=True)
+        run_case(qb, case, BITPLANES, BITPLANES)
+        run_case(qb, case, BITPLANES, INT8, raw=True)
+
+
+@pytest.mark.parametrize("bits", [2, 4])
+def test_config5_square_8192_sampled(qb, bits):
+    """M = N = K = 8192 (compute bound) on the tensor-core path: sampled accumulators and codes."""
+    case = synth.gemm_case(5200 + bits, 8192, 8192, 8192, bits, bits)
+    Wp = qb.pack(qb.to_device_logical(case.W, case.w_enc), bits, case.w_enc, INT8)
+    Ap = qb.pack(qb.to_device_logical(case.At, case.a_enc), bits, case.a_enc, INT8)
+    d = qb.gemm_desc(8192, 8192, 8192, bits, bits, bits, case.w_enc, case.a_enc, INT8, INT8)
+    codes = qb.qgemm(d, Wp, Ap, torch.from_numpy(case.thr).cuda()).cpu().numpy().reshape(8192, 8192)
+    raw = qb.qgemm(d, Wp, Ap, None).cpu().numpy()
+    rng = np.random.default_rng(11)
+    rows = np.concatenate([rng.integers(0, 8192, 2000), [0, 8191, 255, 256]])
+    cols = np.concatenate([rng.integers(0, 8192, 2000), [0, 8191, 127, 128]])
+    acc = orc.dot_at(case.W, case.At, rows, cols)
+    assert np.array_equal(raw[cols, rows].astype(np.int64), acc)
+    want = (acc[:, None] >= case.thr[rows]).sum(axis=1)
+    assert np.array_equal(codes[cols, rows].astype(np.int64), want)
+    full_col = orc.qgemm(case.W, case.At[4321:4322], case.thr)[:, 0]
+    assert np.array_equal(codes[4321, :].astype(np.int64), full_col)
