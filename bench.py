@@ -294,9 +294,120 @@ def run_b200(args):
     qdist.finalize()
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one 4096^3 launch of the tensor-core
-# kernel, from the ncu capture summarised under profiles/ (None until captured).
-TRAFFIC_BYTES_PER_LAUNCH = None
+def _time_calls(torch, fn, iters, warmup=3):
+    """Mean device milliseconds of fn(i), CUDA events on the current stream."""
+    for i in range(warmup):
+        fn(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(iters):
+        fn(warmup + i)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
+def run_extras(args):
+    """The other paper-shaped workloads on one GPU (not the headline line): the large/skinny
+    fully connected sweep (HBM roofline, weight buffers rotated so that every call streams
+    its weights from DRAM), the conv2-shaped layer via lowering, and the AlexNet-shaped
+    chain.  Prints one JSON line."""
+    import torch
+    import __graft_entry__ as ge
+    ge.build()
+    from paper_1709_04060_b200 import binding as qb, synth
+    from paper_1709_04060_b200.alexnet import AlexNetPlan
+    torch.cuda.set_device(0)
+    peaks = load_peaks()
+    PL, I8 = qb.QNN_FMT_BITPLANES, qb.QNN_FMT_INT8
+    res = {"workload": "extras", "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"]}
+
+    # ---- config 5: M = K = 8192, N in {1, 4, 16}; W2A2 and W4A4
+    M = K = 8192
+    skinny = []
+    for bits in (2, 4):
+        c = synth.gemm_case(5000 + bits, M, 16, K, bits, bits)
+        Wd = qb.to_device_logical(c.W, c.w_enc)
+        thr = torch.from_numpy(c.thr).cuda()
+        for fmt, name in ((PL, "bitplanes"), (I8, "int8")):
+            Wp = qb.pack(Wd, bits, c.w_enc, fmt)
+            copies = max(2, int(300e6 // Wp.numel()) + 1)          # > 2 x L2 in rotation
+            Wrot = [Wp] + [Wp.clone() for _ in range(copies - 1)]
+            for N in (1, 4, 16):
+                Ad = qb.to_device_logical(c.At[:N], c.a_enc)
+                Ap = qb.pack(Ad, bits, c.a_enc, fmt)
+                d = qb.gemm_desc(M, N, K, bits, bits, bits, c.w_enc, c.a_enc, fmt, I8)
+                out = torch.empty(qb.qnn_gemm_out_bytes(d, True), dtype=torch.uint8, device="cuda")
+                ms = _time_calls(torch, lambda i: qb.check(qb.qnn_qgemm(d, Wrot[i % copies], Ap, thr, out)), 4 * copies)
+                ms_warm = _time_calls(torch, lambda i: qb.check(qb.qnn_qgemm(d, Wp, Ap, thr, out)), 50)
+                alg = Wp.numel() + Ap.numel() + thr.numel() * 4 + N * M
+                skinny.append({"w": bits, "a": bits, "N": N, "fmt": name, "us": 1e3 * ms, "us_l2_warm": 1e3 * ms_warm,
+                               "algorithmic_bytes": alg, "gbs": alg / ms / 1e6,
+                               "hbm_frac": alg / ms / 1e6 / peaks["hbm_gbs"], "tmacs": M * N * K / ms / 1e9})
+            del Wrot
+    res["skinny_fc"] = skinny
+
+    # ---- config 3: conv2-shaped W1A2 layer via lowering, B = 1 and 64
+    conv = []
+    for B in (1, 64):
+        c = synth.conv2_alexnet_case(B)
+        for fmt, name in ((I8, "int8"), (PL, "bitplanes")):
+            if fmt == PL:
+                x = qb.pack(qb.to_device_logical(c.In.reshape(-1, c.C), c.a_enc), c.a_bits, c.a_enc, PL)
+                pitch = 0
+            else:
+                x = torch.from_numpy(c.In.astype(np.uint8)).cuda()
+                pitch = c.C
+            Wp = qb.pack(qb.to_device_logical(c.Wt.reshape(c.OC, -1), c.w_enc), 1, c.w_enc, fmt)
+            d = qb.qnn_conv_desc(B, 27, 27, 96, pitch, 256, 5, 5, 1, 2, 1, 2, 2, c.w_enc, c.a_enc, fmt, I8, 0)
+            thr = torch.from_numpy(c.thr).cuda()
+            ws = torch.empty(qb.qnn_conv_workspace_bytes(d), dtype=torch.uint8, device="cuda")
+            out = torch.empty(qb.qnn_conv_out_bytes(d, True), dtype=torch.uint8, device="cuda")
+            ms_low = _time_calls(torch, lambda i: qb.check(qb.qnn_im2col(d, x, ws)), 50)
+            ms_all = _time_calls(torch, lambda i: qb.check(qb.qnn_qconv(d, Wp, x, thr, out, ws, ws.numel())), 50)
+            low_bytes = qb.qnn_conv_lowered_bytes(d) + x.numel()
+            conv.append({"B": B, "fmt": name, "im2col_us": 1e3 * ms_low, "im2col_gbs": low_bytes / ms_low / 1e6,
+                         "qconv_us": 1e3 * ms_all, "images_per_s": B / ms_all * 1e3,
+                         "tmacs": B * 729 * 256 * 2400 / ms_all / 1e9})
+    res["conv2"] = conv
+
+    # ---- config 4: AlexNet-shaped chain, B = 1 and 256
+    net_res = []
+    for B in (1, 256):
+        net = synth.alexnet_case(B)
+        for mode in ("tensor", "bitserial") if B == 1 else ("tensor",):
+            plan = AlexNetPlan(net, B, mode)
+            img = torch.from_numpy(net.image.astype(np.uint8)).cuda()
+            ms = _time_calls(torch, lambda i: plan.forward(img), 30 if B == 1 else 10)
+            per_layer = {}
+            for (kind, d, Wp, thr, out), name in zip(plan.steps, plan.names):
+                x_in = img if name == "conv1" else prev
+                if kind == "conv":
+                    f = lambda i: qb.check(qb.qnn_qconv(d, Wp, x_in, thr, out, plan.workspace, plan.workspace.numel()))
+                elif kind == "pool":
+                    f = lambda i: qb.check(qb.qnn_maxpool(d, x_in, out))
+                else:
+                    f = lambda i: qb.check(qb.qnn_qgemm(d, Wp, x_in, thr, out, None, 0))
+                per_layer[name] = round(1e3 * _time_calls(torch, f, 20), 2)
+                prev = out
+            graph, _ = plan.capture(img)
+            ms_graph = _time_calls(torch, lambda i: graph.replay(), 30 if B == 1 else 10)
+            del graph
+            net_res.append({"B": B, "mode": mode, "ms": ms, "images_per_s": B / ms * 1e3,
+                            "ms_graph": ms_graph, "images_per_s_graph": B / ms_graph * 1e3,
+                            "launches": plan.launches_per_forward(), "per_layer_us": per_layer})
+            del plan
+    res["alexnet"] = net_res
+    st, dev = qb.qnn_device_status()
+    assert st == 0 and dev == 0
+    print(json.dumps(res))
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one 4096^3 W1A2 launch of the tensor-core
+# kernel, from the ncu capture summarised in profiles/qgemm_tc_4096_w1a2_w4a4.md (the output
+# codes were still in L2 when the capture ended, so the write counter is small).
+TRAFFIC_BYTES_PER_LAUNCH = 33657856 + 51456
 
 
 def main():
@@ -306,11 +417,16 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="sweep", choices=["sweep", "extras"],
+                    help="sweep: the headline line; extras: the other paper-shaped workloads (one GPU)")
     ap.add_argument("--pairs", default=None,
                     help="restrict the sweep, e.g. '1x2,4x4' (profiling only; the default is all 16)")
     args = ap.parse_args()
     if args.pairs:
         PAIRS[:] = [tuple(int(v) for v in p.split("x")) for p in args.pairs.split(",")]
+    if args.workload == "extras":
+        run_extras(args)
+        return
     if args.impl == "reference":
         if args.steps is None:
             args.steps = 10

@@ -106,6 +106,23 @@ class AlexNetPlan:
             x = out
         return x[: self.B * self.n_classes * 4].view(torch.int32).view(self.B, self.n_classes)
 
+    def capture(self, image: torch.Tensor):
+        """Record one forward pass into a CUDA graph (the chain at small batch is bound by
+        launch overhead, 16 kernels of a few microseconds each).  Returns (graph, logits):
+        ``graph.replay()`` re-runs the chain on the current contents of ``image`` and
+        refreshes ``logits`` in place.  One eager pass runs first so that every one-time
+        set-up of the library happens outside the capture."""
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            self.forward(image)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            logits = self.forward(image)
+        return graph, logits
+
     def intermediates(self):
         """{step name: (output buffer, descriptor kind, descriptor)} for tests."""
         return {n: (s[4], s[0], s[1]) for n, s in zip(self.names, self.steps)}

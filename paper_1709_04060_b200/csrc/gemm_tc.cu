@@ -28,10 +28,18 @@
 // main loop of tile t+1.  Every wait is bounded; on expiry the CTA records
 // QNN_ERR_DEVICE_TIMEOUT in the device status word, drains and exits.
 //
-// Work units: 128 x BN tiles dealt round-robin to the CTAs.  When the last round
-// would fill only part of the GPU, its tiles are cut along the channels into
-// 2, 4 or 8 narrower units (MMA N = BN/2 ..), so that the round costs a fraction of
-// a full tile instead of a whole one.
+// Work units: 128 x BN tiles dealt round-robin to the CTAs.  One MMA costs about the
+// same time for every N (the 128 x 32-byte activation operand is the limit), so a
+// narrower tile is no cheaper; what halves a tile's cost is half the depth.  When the
+// last round would fill at most half of the GPU, the kernel is launched as clusters of
+// two CTAs and each tile of that round is shared by the two CTAs of a cluster, one per
+// half of the depth.  Each CTA then finishes one half of the tile's channels: it stages
+// the int32 partial sums of the other half in its own (by then idle) operand ring and
+// bulk-copies them, 4 KB per 32 x 32 chunk, into the peer's ring (distributed shared
+// memory, completion counted on the peer's mbarriers), while its other four epilogue
+// warps add what the peer sent to their own accumulators and run the threshold
+// epilogue.  Nothing of it touches global memory, and both CTAs of a cluster are
+// resident by construction, so neither can wait for one that is not running.
 #include <cuda.h>
 #include <stdlib.h>
 
@@ -42,11 +50,17 @@ namespace qnn {
 __device__ int g_dev_status;   // QNN_OK or QNN_ERR_DEVICE_TIMEOUT
 
 #ifdef QNN_TC_TRACE
-// Debug builds only: per-tile clock64() stamps of CTA 0, [slot][tile round].
+// Debug builds only: clock64() stamps of one CTA, [slot][unit round].  Slots 0-3: epilogue
+// warp 2 (entry, thresholds ready, accumulators ready, done); 4: CTA start, set-up done, all
+// roles done; 5-7: MMA issuer (accumulator buffer free, first stage landed, all issued);
+// 8: %globaltimer (ns) next to the slot-4 stamps, to convert cycles to time.
 __device__ long long g_trace[16 * 512];
-#define QNN_TRACE(slot, idx) do { if (blockIdx.x == 0 && (idx) < 512) g_trace[(slot) * 512 + (idx)] = clock64(); } while (0)
+__device__ int g_trace_cta;
+#define QNN_TRACE(slot, idx) do { if (blockIdx.x == g_trace_cta && (idx) < 512) g_trace[(slot) * 512 + (idx)] = clock64(); } while (0)
+#define QNN_TRACE_NS(idx) do { if (blockIdx.x == g_trace_cta) { long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_trace[8 * 512 + (idx)] = t_; } } while (0)
 #else
 #define QNN_TRACE(slot, idx) do { } while (0)
+#define QNN_TRACE_NS(idx) do { } while (0)
 #endif
 
 constexpr int TC_BP = 128;          // activation rows (pixels) per tile = tensor-memory lanes
@@ -84,6 +98,41 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
 #pragma unroll 1
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > TC_WAIT_CYCLES) {
+            *abort_flag = 1;
+            atomicExch(&g_dev_status, (int)QNN_ERR_DEVICE_TIMEOUT);
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Bounded wait that also acquires what another CTA of the cluster released on the barrier.
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+    const long long t0 = clock64();
+    for (;;) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.b32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+        if (ok) return true;
         if (*abort_flag) return false;
         if (clock64() - t0 > TC_WAIT_CYCLES) {
             *abort_flag = 1;
@@ -138,27 +187,36 @@ struct TcParams {
     int ld_out;            // INT8 output row pitch
     int fp_count;          // 1: |acc| < 2^22, thresholds are counted on the FP32 pipe
     uint32_t idesc;
-    // work units: [0, full_units) are whole tiles, then every remaining tile is cut
-    // into `split` units of bn_sub channels each
-    int units, full_units, split, bn_sub;
-    uint32_t idesc_sub;
+    // work units: [0, full_units) are whole tiles; unit full_units + 2r + h is half h of
+    // the depth (k-blocks [0, kb_half) / [kb_half, num_kb)) of tile full_units + r
+    int units, full_units, kb_half;
+    int share;             // 1: launched as clusters of two CTAs that share the tiles of the last round
 };
 
-struct TcUnit { int p0, c0, bn; bool sub; };
+// What an epilogue warp needs for the exchange of a shared tile.  The weight ring holds,
+// per lane quarter q, a landing slab (what the peer sends) and a staging slab (what this
+// CTA sends), each [chunk][column / 4][lane] in 16-byte units.
+struct TcExchange {
+    uint32_t zone;         // shared-memory address of the weight ring
+    uint64_t *ring_free;   // the peer's ring is idle (1 arrival from the peer)
+    uint64_t *landed;      // [lane quarter][chunk]: bytes of one chunk from the peer
+    uint32_t rank;         // CTA rank in the cluster = the half of the channels this CTA finishes
+};
 
-__device__ __forceinline__ TcUnit tc_unit(const TcParams &p, int u, int bn_full) {
+struct TcUnit { int p0, c0, kb0, kb1, shared; };   // shared: index of the shared tile, or -1
+
+__device__ __forceinline__ TcUnit tc_unit(const TcParams &p, int u, int bn) {
     TcUnit r;
-    int tile = u, part = 0;
-    r.sub = u >= p.full_units;
-    r.bn = bn_full;
-    if (r.sub) {
+    int tile = u;
+    r.kb0 = 0; r.kb1 = p.num_kb; r.shared = -1;
+    if (u >= p.full_units) {
         const int j = u - p.full_units;
-        tile = p.full_units + j / p.split;
-        part = j - (j / p.split) * p.split;
-        r.bn = p.bn_sub;
+        r.shared = j >> 1;
+        tile = p.full_units + r.shared;
+        if (j & 1) r.kb0 = p.kb_half; else r.kb1 = p.kb_half;
     }
     r.p0 = (tile % p.tiles_p) * TC_BP;
-    r.c0 = (tile / p.tiles_p) * bn_full + part * r.bn;
+    r.c0 = (tile / p.tiles_p) * bn;
     return r;
 }
 
@@ -345,11 +403,62 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams &p, const int *thr
     }
 }
 
+// Exchange of partial sums between the two CTAs of a cluster that share a tile (one per
+// half of the depth); see TcExchange for the layout.
+enum { XCH_NONE = 0, XCH_SEND = 1, XCH_ADD = 2 };
+constexpr uint32_t XCH_CHUNK_BYTES = 32 * 32 * 4;
+
+struct TcXchWarp {
+    int mode;              // XCH_*
+    uint32_t local;        // SEND: staging slab, ADD: landing slab (own shared memory)
+    uint32_t remote;       // SEND: the peer's landing slab (shared::cluster address)
+    uint32_t bars;         // SEND: the peer's landed[q][0] (shared::cluster), ADD: own landed[q][0]
+    volatile int *abort_flag;
+};
+
+// Stage one chunk in own shared memory, then one lane bulk-copies it into the peer's ring;
+// the copy's bytes complete on the peer's barrier of that chunk.
+__device__ __forceinline__ void send_chunk(const TcXchWarp &x, int chunk, const int (&acc)[32], int lane) {
+    const uint32_t src = x.local + (uint32_t)chunk * XCH_CHUNK_BYTES;
+#pragma unroll
+    for (int v = 0; v < 8; ++v)
+        asm volatile("st.shared.v4.s32 [%0], {%1, %2, %3, %4};"
+                     ::"r"(src + (uint32_t)(v * 32 + lane) * 16u), "r"(acc[4 * v]), "r"(acc[4 * v + 1]),
+                       "r"(acc[4 * v + 2]), "r"(acc[4 * v + 3]) : "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // visible to the copy engine
+    __syncwarp();
+    if (lane == 0)
+        asm volatile(
+            "cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+            ::"r"(x.remote + (uint32_t)chunk * XCH_CHUNK_BYTES), "r"(src), "r"(XCH_CHUNK_BYTES),
+              "r"(x.bars + (uint32_t)chunk * 8u) : "memory");
+}
+// Wait for the peer's chunk and add it.  Returns false if the wait ran out.
+__device__ __forceinline__ bool add_chunk(const TcXchWarp &x, int chunk, int (&acc)[32], int lane) {
+    bool ok = true;
+    if (lane == 0)
+        ok = mbar_wait_cluster(reinterpret_cast<uint64_t *>(__cvta_shared_to_generic(x.bars + (uint32_t)chunk * 8u)),
+                               0, x.abort_flag);
+    ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+    __syncwarp();
+    if (!ok) return false;
+    const uint32_t src = x.local + (uint32_t)chunk * XCH_CHUNK_BYTES;
+#pragma unroll
+    for (int v = 0; v < 8; ++v) {
+        int a, b, c, d;
+        asm volatile("ld.shared.v4.s32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(a), "=r"(b), "=r"(c), "=r"(d) : "r"(src + (uint32_t)(v * 32 + lane) * 16u) : "memory");
+        acc[4 * v] += a; acc[4 * v + 1] += b; acc[4 * v + 2] += c; acc[4 * v + 3] += d;
+    }
+    return true;
+}
+
 // Columns [c_begin, c_end) of one accumulator tile for this thread's pixel.  The
 // tensor-memory load of the next chunk is in flight while the current one is processed.
 template <int OUT_MODE, int OUT_BITS>
 __device__ __forceinline__ void epilogue_cols(const TcParams &p, const int *thr_s, uint32_t t_row,
-                                              int c_begin, int c_end, int n, int m0) {
+                                              int c_begin, int c_end, int n, int m0, const TcXchWarp &x,
+                                              int lane) {
     constexpr int NT = thr_slots(OUT_BITS);
     int c_stop = c_end;                                  // skip chunks wholly beyond M (warp-uniform)
     if (m0 + c_stop > p.M) c_stop = c_begin + ((p.M - m0 - c_begin + 31) & ~31);
@@ -362,11 +471,21 @@ __device__ __forceinline__ void epilogue_cols(const TcParams &p, const int *thr_
         tmem_ld_wait(acc_a);
         const bool has_b = c0 + 32 < c_stop;
         if (has_b) tmem_ld32_issue(t_row + c0 + 32, acc_b);
-        epilogue_chunk<OUT_MODE, OUT_BITS>(p, thr_s + c0 * NT, acc_a, n, n_ok, m0 + c0);
+        if (x.mode == XCH_SEND) {
+            send_chunk(x, (c0 - c_begin) >> 5, acc_a, lane);
+        } else {
+            if (x.mode == XCH_ADD && !add_chunk(x, (c0 - c_begin) >> 5, acc_a, lane)) return;
+            epilogue_chunk<OUT_MODE, OUT_BITS>(p, thr_s + c0 * NT, acc_a, n, n_ok, m0 + c0);
+        }
         if (has_b) {
             tmem_ld_wait(acc_b);
             if (c0 + 64 < c_stop) tmem_ld32_issue(t_row + c0 + 64, acc_a);
-            epilogue_chunk<OUT_MODE, OUT_BITS>(p, thr_s + (c0 + 32) * NT, acc_b, n, n_ok, m0 + c0 + 32);
+            if (x.mode == XCH_SEND) {
+                send_chunk(x, (c0 + 32 - c_begin) >> 5, acc_b, lane);
+            } else {
+                if (x.mode == XCH_ADD && !add_chunk(x, (c0 + 32 - c_begin) >> 5, acc_b, lane)) return;
+                epilogue_chunk<OUT_MODE, OUT_BITS>(p, thr_s + (c0 + 32) * NT, acc_b, n, n_ok, m0 + c0 + 32);
+            }
         }
     }
 }
@@ -401,7 +520,8 @@ template <int OUT_MODE, int OUT_BITS>
 __device__ __forceinline__ bool epilogue_tile(const TcParams &p, const int *thr_s, uint64_t *thr_full,
                                               uint64_t *thr_empty, uint32_t thr_parity,
                                               uint64_t *tmem_full, uint32_t full_parity,
-                                              uint32_t t_acc, int bn, int p0, int c0, int warp, int lane,
+                                              uint32_t t_acc, int bn, int p0, int c0, int shared,
+                                              const TcExchange &x, int warp, int lane,
                                               volatile int *abort_flag, int full_parity_dbg = 0) {
     const int quad = warp & 3, half = (warp - 2) >> 2;
     const bool tr = warp == 2 && lane == 0;
@@ -413,8 +533,35 @@ __device__ __forceinline__ bool epilogue_tile(const TcParams &p, const int *thr_
     tc_fence_after();
     const int hcols = bn >= 64 ? bn / 2 : bn;
     const int c_begin = half * hcols, c_end = (bn >= 64 || half == 0) ? c_begin + hcols : c_begin;
+    TcXchWarp xw;
+    xw.mode = XCH_NONE; xw.local = xw.remote = xw.bars = 0; xw.abort_flag = abort_flag;
+    if (shared >= 0) {
+        // warps whose channel half equals the CTA's rank finish those channels; the others
+        // send their half to the peer, whose rank it equals
+        const uint32_t peer = x.rank ^ 1u;
+        const uint32_t slab_bytes = (uint32_t)hcols * 128u;            // hcols columns x 32 lanes x 4 bytes
+        const int chunks = hcols >> 5;
+        // all MMAs of this CTA are complete: its operand ring may be overwritten
+        if (warp == 2 && lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(x.ring_free), peer));
+        if ((uint32_t)half == x.rank) {
+            xw.mode = XCH_ADD;
+            xw.local = x.zone + (uint32_t)quad * slab_bytes;
+            xw.bars = smem_u32(&x.landed[quad * 4]);
+            if (lane == 0)
+                for (int c = 0; c < chunks; ++c) mbar_arrive_expect_tx(&x.landed[quad * 4 + c], XCH_CHUNK_BYTES);
+        } else {
+            bool ok = true;
+            if (lane == 0) ok = mbar_wait_cluster(x.ring_free, 0, abort_flag);
+            if (__shfl_sync(0xffffffffu, (int)ok, 0) == 0) return false;
+            __syncwarp();
+            xw.mode = XCH_SEND;
+            xw.local = x.zone + (uint32_t)(4 + quad) * slab_bytes;
+            xw.remote = map_to_cta(x.zone + (uint32_t)quad * slab_bytes, peer);
+            xw.bars = map_to_cta(smem_u32(&x.landed[quad * 4]), peer);
+        }
+    }
     epilogue_cols<OUT_MODE, OUT_BITS>(p, thr_s, t_acc + ((uint32_t)(quad * 32) << 16), c_begin, c_end,
-                                      p0 + quad * 32 + lane, c0);
+                                      p0 + quad * 32 + lane, c0, xw, lane);
     tc_fence_before();
     __syncwarp();
     if (OUT_MODE != OUT_RAW && lane == 0) mbar_arrive(thr_empty);
@@ -434,6 +581,8 @@ struct TcSmem {
     uint64_t tmem_empty[2];
     uint64_t thr_full[2];
     uint64_t thr_empty[2];
+    uint64_t ring_free;
+    uint64_t landed[4 * 4];
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -441,14 +590,16 @@ struct TcSmem {
 template <int BN, int STAGES, int OUT_MODE, int OUT_BITS>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_constant__ CUtensorMap map_wgt,
-                const __grid_constant__ CUtensorMap map_wgt_sub, const TcParams p) {
+                const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
     using Smem = TcSmem<BN, STAGES, OUT_BITS>;
     Smem &sm = *reinterpret_cast<Smem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     constexpr uint32_t TMEM_COLS = (2 * BN < 32) ? 32 : 2 * BN;
+    constexpr uint32_t STAGE_BYTES = (TC_BP + BN) * TC_BK;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int *abort_flag = &sm.abort_flag;
+    if (threadIdx.x == 0) { QNN_TRACE(4, 0); QNN_TRACE_NS(0); }
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
@@ -456,14 +607,18 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
             mbar_init(&sm.tmem_full[b], 1); mbar_init(&sm.tmem_empty[b], EPI_WARPS);
             mbar_init(&sm.thr_full[b], 1); mbar_init(&sm.thr_empty[b], EPI_WARPS);
         }
+        mbar_init(&sm.ring_free, 1);
+        for (int e = 0; e < 16; ++e) mbar_init(&sm.landed[e], 1);
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) tmem_alloc(&sm.tmem_base, TMEM_COLS);
     tc_fence_before();
-    __syncthreads();
+    if (p.share) cluster_sync_all();       // the peer's barriers are initialised before anyone signals them
+    else __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = sm.tmem_base;
+    if (threadIdx.x == 0) QNN_TRACE(4, 1);
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
@@ -472,15 +627,13 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
             bool ok = true;
             for (int u = blockIdx.x; ok && u < p.units; u += gridDim.x) {
                 const TcUnit un = tc_unit(p, u, BN);
-                const CUtensorMap *mw = un.sub ? &map_wgt_sub : &map_wgt;
-                const uint32_t stage_bytes = (uint32_t)(TC_BP + un.bn) * TC_BK;
-                for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
+                for (int kb = un.kb0; kb < un.kb1; ++kb, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1;
                     if (!(ok = mbar_wait(&sm.empty[s], ph ^ 1, abort_flag))) break;
-                    mbar_arrive_expect_tx(&sm.full[s], stage_bytes);
+                    mbar_arrive_expect_tx(&sm.full[s], STAGE_BYTES);
                     tma_load_2d(sm.act[s], &map_act, &sm.full[s], kb * TC_BK, un.p0);
-                    tma_load_2d(sm.wgt[s], mw, &sm.full[s], kb * TC_BK, un.c0);
+                    tma_load_2d(sm.wgt[s], &map_wgt, &sm.full[s], kb * TC_BK, un.c0);
                 }
             }
             if (!ok) {
@@ -497,23 +650,26 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
             bool ok = true;
             for (int u = blockIdx.x; ok && u < p.units; u += gridDim.x, ++tcount) {
                 const uint32_t buf = tcount & 1, acc_ph = (tcount >> 1) & 1;
-                const uint32_t idesc = u >= p.full_units ? p.idesc_sub : p.idesc;
+                const TcUnit un = tc_unit(p, u, BN);
                 if (!(ok = mbar_wait(&sm.tmem_empty[buf], acc_ph ^ 1, abort_flag))) break;
                 tc_fence_after();
+                QNN_TRACE(5, tcount);
                 const uint32_t d_tmem = tmem_base + buf * BN;
-                for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
+                for (int kb = un.kb0; kb < un.kb1; ++kb, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1;
                     if (!(ok = mbar_wait(&sm.full[s], ph, abort_flag))) break;
                     tc_fence_after();
+                    if (kb == un.kb0) QNN_TRACE(6, tcount);
                     const uint64_t da = umma_smem_desc(smem_u32(sm.act[s]));
                     const uint64_t db = umma_smem_desc(smem_u32(sm.wgt[s]));
 #pragma unroll
                     for (int kk = 0; kk < TC_BK / 32; ++kk)   // 32 depth bytes per MMA: +2 in 16-byte units
-                        umma_i8(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (kb | kk) != 0);
+                        umma_i8(d_tmem, da + 2 * kk, db + 2 * kk, p.idesc, (kb > un.kb0) || kk != 0);
                     umma_commit(&sm.empty[s]);
                 }
                 if (ok) umma_commit(&sm.tmem_full[buf]);
+                QNN_TRACE(7, tcount);
             }
         }
         __syncwarp();
@@ -525,25 +681,31 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
                                           const long long u = blockIdx.x + (long long)i * gridDim.x;
                                           if (u >= p.units) return false;
                                           const TcUnit un = tc_unit(p, (int)u, BN);
-                                          c0 = un.c0; bn = un.bn;
+                                          c0 = un.c0; bn = BN;
                                           return true;
                                       });
     } else {
         // ------------------------------------------------------------ epilogue
         uint32_t tcount = 0;
+        TcExchange xc;
+        xc.zone = smem_u32(&sm.wgt[0][0]);
+        xc.ring_free = &sm.ring_free; xc.landed = sm.landed;
+        xc.rank = p.share ? cluster_ctarank() : 0u;
         for (int u = blockIdx.x; u < p.units; u += gridDim.x, ++tcount) {
             const TcUnit un = tc_unit(p, u, BN);
             const uint32_t buf = tcount & 1, acc_ph = (tcount >> 1) & 1;
             if (!epilogue_tile<OUT_MODE, OUT_BITS>(p, sm.thr[buf], &sm.thr_full[buf], &sm.thr_empty[buf], acc_ph,
-                                                   &sm.tmem_full[buf], acc_ph, tmem_base + buf * BN, un.bn,
-                                                   un.p0, un.c0, warp, lane, abort_flag, (int)tcount))
+                                                   &sm.tmem_full[buf], acc_ph, tmem_base + buf * BN, BN,
+                                                   un.p0, un.c0, un.shared, xc, warp, lane, abort_flag, (int)tcount))
                 break;
             if (lane == 0) mbar_arrive(&sm.tmem_empty[buf]);     // one arrival per warp
         }
     }
 
     tc_fence_before();
-    __syncthreads();
+    if (p.share) cluster_sync_all();       // the peer may still write this CTA's shared memory or barriers
+    else __syncthreads();
+    if (threadIdx.x == 0) { QNN_TRACE(4, 2); QNN_TRACE_NS(2); }
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
@@ -575,22 +737,6 @@ struct Tc2Smem {
     int abort_flag;
 };
 
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
 __device__ __forceinline__ void tma_load_2d_pair(void *dst, const CUtensorMap *map, uint32_t bar_cluster_addr,
                                                  int x, int y) {
     asm volatile(
@@ -719,7 +865,7 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_const
             const uint32_t buf = tcount & 1, acc_ph = (tcount >> 1) & 1;
             if (!epilogue_tile<OUT_MODE, OUT_BITS>(p, sm.thr[buf], &sm.thr_full[buf], &sm.thr_empty[buf], acc_ph,
                                                    &sm.tmem_full[buf], acc_ph, tmem_base + buf * T2_BN, T2_BN,
-                                                   p0, c0, warp, lane, abort_flag))
+                                                   p0, c0, -1, TcExchange{}, warp, lane, abort_flag))
                 break;
             if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&sm.tmem_empty[buf]), 0));
         }
@@ -766,8 +912,7 @@ static bool make_map(CUtensorMap *map, const void *base, int rows, int K, int ld
 }
 
 template <int BN, int STAGES, int OUT_MODE, int OUT_BITS>
-static qnn_status launch_cfg(const CUtensorMap &ma, const CUtensorMap &mw, const CUtensorMap &mws,
-                             const TcParams &p, cudaStream_t s) {
+static qnn_status launch_cfg(const CUtensorMap &ma, const CUtensorMap &mw, const TcParams &p, cudaStream_t s) {
     auto kern = qgemm_tc_kernel<BN, STAGES, OUT_MODE, OUT_BITS>;
     const size_t smem = sizeof(TcSmem<BN, STAGES, OUT_BITS>) + 1024;
     static bool attr_done = false;        // per instantiation
@@ -777,7 +922,19 @@ static qnn_status launch_cfg(const CUtensorMap &ma, const CUtensorMap &mw, const
         attr_done = true;
     }
     const int grid = p.units < sm_count() ? p.units : sm_count();
-    kern<<<grid, TC_THREADS, smem, s>>>(ma, mw, mws, p);
+    if (p.share) {
+        // clusters of two CTAs: consecutive block indices share a tile of the last round
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid); cfg.blockDim = dim3(TC_THREADS);
+        cfg.dynamicSmemBytes = smem; cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, kern, ma, mw, p) != cudaSuccess) return QNN_ERR_CUDA;
+    } else {
+        kern<<<grid, TC_THREADS, smem, s>>>(ma, mw, p);
+    }
     count_launch();
     return launch_status();
 }
@@ -812,8 +969,8 @@ static qnn_status launch_pair_cfg(const CUtensorMap &ma, const CUtensorMap &mw, 
 
 template <int BN, int STAGES>
 static qnn_status launch_out(int mode, int out_bits, const CUtensorMap &ma, const CUtensorMap &mw,
-                             const CUtensorMap &mws, const TcParams &p, cudaStream_t s) {
-#define QNN_C1(MODE_, BITS_) launch_cfg<BN, STAGES, MODE_, BITS_>(ma, mw, mws, p, s)
+                             const TcParams &p, cudaStream_t s) {
+#define QNN_C1(MODE_, BITS_) launch_cfg<BN, STAGES, MODE_, BITS_>(ma, mw, p, s)
     QNN_TC_DISPATCH(QNN_C1(OUT_RAW, 0), QNN_C1)
 #undef QNN_C1
 }
@@ -833,6 +990,32 @@ static bool choose_pair_kernel(const qnn_gemm_desc *d, int sms) {
     return false;
 }
 
+// Tile plan of the one-CTA kernel: channel tile, grid, and whether the tiles of the last
+// round are shared by the CTA pairs of two-CTA clusters.
+struct TcPlan {
+    int bn, tiles_p, tiles_c, grid, rem;
+    bool share;
+};
+
+static bool tc_plan(const qnn_gemm_desc *d, int sms, TcPlan *pl) {
+    // channel tile: the widest that still gives every SM a tile
+    const int tiles_p = ceil_div(d->N, TC_BP);
+    int bn = 256;
+    while (bn > 32 && (bn / 2 >= round_up(d->M, 32) || (long long)tiles_p * ceil_div(d->M, bn) < sms)) bn >>= 1;
+    if (bn == 64) bn = 32;
+    pl->bn = bn; pl->tiles_p = tiles_p; pl->tiles_c = ceil_div(d->M, bn);
+    const long long tiles = (long long)pl->tiles_p * pl->tiles_c;
+    if (tiles > 0x3fffffff) return false;
+    pl->grid = tiles < sms ? (int)tiles : sms;
+    pl->rem = (int)(tiles % pl->grid);
+    // sharing: a partial last round on at most half of an even number of SMs; the landing
+    // zone is the weight ring (bn x 512 bytes of sums fit STAGES >= 4 stages of bn x 128 bytes)
+    const char *no_share = getenv("QNN_TC_NO_SHARE");
+    pl->share = pl->rem > 0 && 2 * pl->rem <= pl->grid && (pl->grid % 2) == 0 && bn >= 128 &&
+                ceil_div(d->K, TC_BK) >= 2 && !(no_share && no_share[0] == '1');
+    return true;
+}
+
 qnn_status gemm_tc_launch(const qnn_gemm_desc *d, const void *W, const void *A, const int32_t *thr,
                           void *out, cudaStream_t s) {
     const int ld = round_up(d->K, 16);
@@ -843,6 +1026,7 @@ qnn_status gemm_tc_launch(const qnn_gemm_desc *d, const void *W, const void *A, 
     p.thr = thr; p.out = out; p.M = d->M; p.N = d->N; p.K = d->K;
     p.num_kb = ceil_div(d->K, TC_BK);
     p.ld_out = round_up(d->M, 16);
+    p.kb_half = 0; p.share = 0;
     const double wmax = d->w_enc == QNN_ENC_BIPOLAR ? 1.0
                         : (d->w_enc == QNN_ENC_SIGNED ? double(1 << (d->w_bits - 1)) : double((1 << d->w_bits) - 1));
     const double amax = d->a_enc == QNN_ENC_BIPOLAR ? 1.0
@@ -859,44 +1043,37 @@ qnn_status gemm_tc_launch(const qnn_gemm_desc *d, const void *W, const void *A, 
     if (pair) {
         if (!make_map(&ma, A, d->N, d->K, ld, TC_BP) || !make_map(&mw, W, d->M, d->K, ld, 128)) return QNN_ERR_CUDA;
         p.tiles_p = ceil_div(d->N, 256); p.tiles_c = ceil_div(d->M, T2_BN);
-        p.units = p.full_units = p.tiles_p * p.tiles_c; p.split = 1; p.bn_sub = T2_BN; p.idesc_sub = 0;
+        p.units = p.full_units = p.tiles_p * p.tiles_c;
         p.idesc = idesc_base | ((uint32_t)(T2_BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
         return launch_pair_out(mode, d->out_bits, ma, mw, p, s);
     }
-    // channel tile: the widest that still gives every SM a tile
-    const int tiles_p = ceil_div(d->N, TC_BP);
-    int bn = 256;
-    while (bn > 32 && (bn / 2 >= round_up(d->M, 32) || (long long)tiles_p * ceil_div(d->M, bn) < sms)) bn >>= 1;
-    if (bn == 64) bn = 32;
-    p.tiles_p = tiles_p; p.tiles_c = ceil_div(d->M, bn);
-    // Work units: when the last round of tiles would occupy at most half of the SMs, cut
-    // each of its tiles along the channels so that the round costs 1/split of a tile.
-    const long long tiles = (long long)p.tiles_p * p.tiles_c;
-    if (tiles > 0x3fffffff) return QNN_ERR_UNSUPPORTED;
-    const int grid = tiles < sms ? (int)tiles : sms;
-    const int rem = (int)(tiles % grid);
-    int split = 1;
-    if (rem > 0)
-        while (2 * split * rem <= grid && bn / (2 * split) >= 32) split *= 2;
-    p.split = split; p.bn_sub = bn / split;
-    p.full_units = split > 1 ? (int)tiles - rem : (int)tiles;
-    p.units = p.full_units + (split > 1 ? rem * split : 0);
+    TcPlan pl;
+    if (!tc_plan(d, sms, &pl)) return QNN_ERR_UNSUPPORTED;
+    const int bn = pl.bn;
+    p.tiles_p = pl.tiles_p; p.tiles_c = pl.tiles_c;
+    const int tiles = pl.tiles_p * pl.tiles_c;
+    p.units = p.full_units = tiles;
+    if (pl.share) {
+        p.share = 1;
+        p.full_units = tiles - pl.rem;
+        p.units = p.full_units + 2 * pl.rem;
+        p.kb_half = (p.num_kb + 1) / 2;
+    }
     p.idesc = idesc_base | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(TC_BP >> 4) << 24);
-    p.idesc_sub = idesc_base | ((uint32_t)(p.bn_sub >> 3) << 17) | ((uint32_t)(TC_BP >> 4) << 24);
-    CUtensorMap mws;
-    if (!make_map(&ma, A, d->N, d->K, ld, TC_BP) || !make_map(&mw, W, d->M, d->K, ld, bn) ||
-        !make_map(&mws, W, d->M, d->K, ld, p.bn_sub))
-        return QNN_ERR_CUDA;
+    if (!make_map(&ma, A, d->N, d->K, ld, TC_BP) || !make_map(&mw, W, d->M, d->K, ld, bn)) return QNN_ERR_CUDA;
     switch (bn) {
-        case 256: return launch_out<256, 4>(mode, d->out_bits, ma, mw, mws, p, s);
-        case 128: return launch_out<128, 6>(mode, d->out_bits, ma, mw, mws, p, s);
-        default:  return launch_out<32, 8>(mode, d->out_bits, ma, mw, mws, p, s);
+        case 256: return launch_out<256, 4>(mode, d->out_bits, ma, mw, p, s);
+        case 128: return launch_out<128, 6>(mode, d->out_bits, ma, mw, p, s);
+        default:  return launch_out<32, 8>(mode, d->out_bits, ma, mw, p, s);
     }
 }
 
 #ifdef QNN_TC_TRACE
 extern "C" int qnn_debug_read_trace(long long *host, int n) {
     return (int)cudaMemcpyFromSymbol(host, g_trace, sizeof(long long) * n);
+}
+extern "C" int qnn_debug_trace_cta(int cta) {
+    return (int)cudaMemcpyToSymbol(g_trace_cta, &cta, sizeof(int));
 }
 #endif
 

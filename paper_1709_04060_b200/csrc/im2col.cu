@@ -108,6 +108,56 @@ __global__ void __launch_bounds__(256) lower_bytes_kernel(const LowerParams p) {
     }
 }
 
+// Byte-granular lowering through shared memory: a CTA takes LB_PIX consecutive output
+// pixels of one output row, stages the KH input-row segments they touch (compact, C bytes
+// per pixel, zeros outside the image) and then assembles the lowered rows from shared
+// memory, one warp per output pixel, 4 bytes per lane and step, with coalesced stores.
+constexpr int LB_PIX = 32;
+
+__global__ void __launch_bounds__(256) lower_bytes_smem_kernel(const LowerParams p, int chunks, int span) {
+    extern __shared__ uint8_t lb_smem[];                 // [KH][span * C]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint8_t *in = reinterpret_cast<const uint8_t *>(p.in);
+    uint32_t *out = reinterpret_cast<uint32_t *>(p.out);
+    const int row_words = p.row_units >> 2;
+    const int seg_bytes = span * p.cu;                   // bytes of one staged input-row segment
+    const long long jobs = (long long)p.B * p.OH * chunks;
+    for (long long job = blockIdx.x; job < jobs; job += gridDim.x) {
+        const int chunk = (int)(job % chunks);
+        const long long t = job / chunks;
+        const int oh = (int)(t % p.OH), b = (int)(t / p.OH);
+        const int ow0 = chunk * LB_PIX;
+        const int npx = min(LB_PIX, p.OW - ow0);
+        const int ih0 = oh * p.stride - p.pad, iw0 = ow0 * p.stride - p.pad;
+        __syncthreads();                                 // previous job's readers are done
+        for (int e = threadIdx.x; e < p.KH * seg_bytes; e += blockDim.x) {
+            const int kh = e / seg_bytes, r = e - kh * seg_bytes;
+            const int px = (int)fdiv((uint32_t)r, p.cud), c = r - px * p.cu;
+            const int ih = ih0 + kh, iw = iw0 + px;
+            uint8_t v = 0;
+            if (ih >= 0 && ih < p.H && iw >= 0 && iw < p.W)
+                v = in[(((size_t)b * p.H + ih) * p.W + iw) * p.pitch + c];
+            lb_smem[e] = v;
+        }
+        __syncthreads();
+        for (int px = warp; px < npx; px += 8) {
+            const uint8_t *src = lb_smem + px * p.stride * p.cu;
+            uint32_t *dst = out + (((size_t)b * p.OH + oh) * p.OW + ow0 + px) * row_words;
+            for (int q = lane; q < row_words; q += 32) {
+                int k = q * 4;
+                int kh = (int)fdiv((uint32_t)k, p.seg), r = k - kh * (int)p.seg.d;
+                uint32_t v = 0;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if (k + e < p.row_copy) v |= (uint32_t)src[kh * seg_bytes + r] << (8 * e);
+                    if (++r == (int)p.seg.d) { r = 0; ++kh; }
+                }
+                dst[q] = v;
+            }
+        }
+    }
+}
+
 qnn_status im2col_launch(const qnn_conv_desc *d, const void *in, void *lowered, cudaStream_t s) {
     LowerParams p;
     p.in = in; p.out = lowered;
@@ -148,6 +198,19 @@ qnn_status im2col_launch(const qnn_conv_desc *d, const void *in, void *lowered, 
     const long long jobs = p.npix * p.planes;
     long long blocks = (jobs * 32 + threads - 1) / threads;
     if (blocks > max_blocks) blocks = max_blocks;
+    if (mode == 2) {
+        // staged variant when the input-row segments of 32 output pixels fit 48 KB
+        const int span = (LB_PIX - 1) * d->stride + d->KW;
+        const size_t smem = (size_t)d->KH * span * p.cu;
+        if (smem <= 48 * 1024 && smem < (1u << 24)) {
+            const int chunks = ceil_div(p.OW, LB_PIX);
+            long long nb = (long long)d->B * p.OH * chunks;
+            if (nb > max_blocks) nb = max_blocks;
+            lower_bytes_smem_kernel<<<(unsigned)nb, threads, smem, s>>>(p, chunks, span);
+            count_launch();
+            return launch_status();
+        }
+    }
     if (mode == 0) lower_units_kernel<uint32_t><<<(unsigned)blocks, threads, 0, s>>>(p);
     else if (mode == 1) lower_units_kernel<uint4><<<(unsigned)blocks, threads, 0, s>>>(p);
     else lower_bytes_kernel<<<(unsigned)blocks, threads, 0, s>>>(p);

@@ -192,3 +192,22 @@ def test_alexnet_chain_per_layer(qb, mode, B):
         got = decode_out(buf.cpu().numpy(), fmt, 2, npix, C, False)
         assert np.array_equal(got, want.reshape(npix, C)), f"{mode}: first mismatch after {L.name}"
     assert np.array_equal(logits.cpu().numpy().astype(np.int64), logits_ref)
+
+
+def test_alexnet_chain_graph_replay(qb):
+    """The chain recorded into a CUDA graph gives the oracle's logits on replay, also after
+    the input buffer has been overwritten with another batch."""
+    from paper_1709_04060_b200.alexnet import AlexNetPlan
+    net_a, net_b = synth.alexnet_case(2, seed=4), synth.alexnet_case(2, seed=5)
+    net_b.weights, net_b.thr = net_a.weights, net_a.thr          # same network, other images
+    plan = AlexNetPlan(net_a, 2, "tensor")
+    img = torch.from_numpy(net_a.image.astype(np.uint8)).cuda()
+    graph, logits = plan.capture(img)
+    for net in (net_a, net_b, net_a):
+        img.copy_(torch.from_numpy(net.image.astype(np.uint8)))
+        graph.replay()
+        torch.cuda.synchronize()
+        want, _ = onet.forward(net, keep_intermediates=False)
+        assert np.array_equal(logits.cpu().numpy().astype(np.int64), want)
+    st, dev = qb.qnn_device_status()
+    assert st == 0 and dev == 0

@@ -159,17 +159,29 @@ def test_both_tensor_core_kernels(qb, force_tc_kernel, which, M, N, K, w, a):
 
 
 @pytest.mark.parametrize("M,N,K,w,a", [
-    (250, 19195, 256, 1, 2),     # 150 tiles on 148 SMs: the last 2 are cut into 8 units of 32 channels
-    (512, 10240, 160, 2, 4),     # 160 tiles: the last 12 are cut into 4 units of 64 channels
-    (768, 8440, 192, 4, 3),      # 198 tiles: the last 50 are cut into 2 units of 128 channels
+    (250, 19195, 256, 1, 2),     # 150 tiles on 148 SMs: the last 2 are shared, 1 + 1 k-blocks
+    (512, 10240, 160, 2, 4),     # 160 tiles: the last 12 are shared (two k-blocks, the second ragged)
+    (768, 8440, 1100, 4, 3),     # 198 tiles: the last 50 are shared, 5 + 4 k-blocks
 ])
-def test_partial_last_round_is_cut_into_narrow_units(qb, M, N, K, w, a):
-    """Tile counts just above a multiple of the SM count: the tiles of the last round are
-    split along the channels (narrower MMAs, second weight tensor map); every output checked."""
+def test_partial_last_round_is_shared_by_cta_pairs(qb, monkeypatch, M, N, K, w, a):
+    """Tile counts just above a multiple of the SM count: the kernel runs as two-CTA clusters
+    and each tile of the last round is computed by the two CTAs of a cluster, half of the
+    depth each; the odd CTA hands its int32 partial sums to the even one through distributed
+    shared memory before the threshold epilogue.  Every output is checked, and the same
+    problem with sharing switched off must give identical bytes."""
     case = synth.gemm_case(1200 + M, M, N, K, w, a)
     run_case(qb, case, INT8, INT8)
     run_case(qb, case, INT8, BITPLANES)
     run_case(qb, case, INT8, INT8, raw=True)
+    d = qb.gemm_desc(M, N, K, w, a, case.out_bits, case.w_enc, case.a_enc, INT8, INT8)
+    Wp = qb.pack(qb.to_device_logical(case.W, case.w_enc), w, case.w_enc, INT8)
+    Ap = qb.pack(qb.to_device_logical(case.At, case.a_enc), a, case.a_enc, INT8)
+    thr = torch.from_numpy(case.thr).cuda()
+    shared = qb.qgemm(d, Wp, Ap, thr).clone()
+    monkeypatch.setenv("QNN_TC_NO_SHARE", "1")
+    whole = qb.qgemm(d, Wp, Ap, thr)
+    torch.cuda.synchronize()
+    assert torch.equal(shared, whole)
 
 
 @pytest.mark.parametrize("which", ["single", "pair"])
