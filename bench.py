@@ -385,6 +385,8 @@ def run_extras(args):
                 x_in = img if name == "conv1" else prev
                 if kind == "conv":
                     f = lambda i: qb.check(qb.qnn_qconv(d, Wp, x_in, thr, out, plan.workspace, plan.workspace.numel()))
+                    per_layer[name + "_lowering"] = round(
+                        1e3 * _time_calls(torch, lambda i: qb.check(qb.qnn_im2col(d, x_in, plan.workspace)), 20), 2)
                 elif kind == "pool":
                     f = lambda i: qb.check(qb.qnn_maxpool(d, x_in, out))
                 else:

@@ -115,12 +115,15 @@ __global__ void __launch_bounds__(256) lower_bytes_kernel(const LowerParams p) {
 constexpr int LB_PIX = 32;
 
 __global__ void __launch_bounds__(256) lower_bytes_smem_kernel(const LowerParams p, int chunks, int span) {
-    extern __shared__ uint8_t lb_smem[];                 // [KH][span * C]
+    extern __shared__ __align__(16) uint8_t lb_smem[];   // [KH][seg_pitch], seg_pitch = span * C rounded up to 4
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint8_t *in = reinterpret_cast<const uint8_t *>(p.in);
     uint32_t *out = reinterpret_cast<uint32_t *>(p.out);
+    const uint32_t *sm_words = reinterpret_cast<const uint32_t *>(lb_smem);
     const int row_words = p.row_units >> 2;
     const int seg_bytes = span * p.cu;                   // bytes of one staged input-row segment
+    const int seg_pitch = (seg_bytes + 3) & ~3;
+    const int tap_bytes = (int)p.seg.d;                  // KW * C: bytes one filter row contributes
     const long long jobs = (long long)p.B * p.OH * chunks;
     for (long long job = blockIdx.x; job < jobs; job += gridDim.x) {
         const int chunk = (int)(job % chunks);
@@ -130,29 +133,50 @@ __global__ void __launch_bounds__(256) lower_bytes_smem_kernel(const LowerParams
         const int npx = min(LB_PIX, p.OW - ow0);
         const int ih0 = oh * p.stride - p.pad, iw0 = ow0 * p.stride - p.pad;
         __syncthreads();                                 // previous job's readers are done
-        for (int e = threadIdx.x; e < p.KH * seg_bytes; e += blockDim.x) {
-            const int kh = e / seg_bytes, r = e - kh * seg_bytes;
-            const int px = (int)fdiv((uint32_t)r, p.cud), c = r - px * p.cu;
-            const int ih = ih0 + kh, iw = iw0 + px;
-            uint8_t v = 0;
-            if (ih >= 0 && ih < p.H && iw >= 0 && iw < p.W)
-                v = in[(((size_t)b * p.H + ih) * p.W + iw) * p.pitch + c];
-            lb_smem[e] = v;
+        // stage: one warp per filter row, lanes along the bytes of the segment
+        for (int kh = warp; kh < p.KH; kh += 8) {
+            const int ih = ih0 + kh;
+            const bool row_ok = ih >= 0 && ih < p.H;
+            const uint8_t *row = in + (((size_t)b * p.H + (row_ok ? ih : 0)) * p.W) * p.pitch;
+            uint8_t *dst = lb_smem + kh * seg_pitch;
+            if (p.pitch == p.cu) {
+                // pixels are contiguous: byte r of the segment is byte iw0*C + r of the image row
+                const int lo = max(0, -iw0) * p.cu, hi = min(span, p.W - iw0) * p.cu;
+                const uint8_t *src = row + (long long)iw0 * p.cu;
+                for (int r = lane; r < seg_pitch; r += 32)
+                    dst[r] = (row_ok && r >= lo && r < hi) ? src[r] : (uint8_t)0;
+            } else {
+                for (int r = lane; r < seg_pitch; r += 32) {
+                    const int px = (int)fdiv((uint32_t)r, p.cud), c = r - px * p.cu;
+                    const int iw = iw0 + px;
+                    dst[r] = (row_ok && r < seg_bytes && iw >= 0 && iw < p.W) ? row[(size_t)iw * p.pitch + c]
+                                                                               : (uint8_t)0;
+                }
+            }
         }
         __syncthreads();
+        // assemble: within one filter row the bytes of a lowered row are contiguous in the
+        // staged segment, so a word is an unaligned 4-byte read (two aligned words and a
+        // funnel shift) unless it straddles two filter rows
         for (int px = warp; px < npx; px += 8) {
-            const uint8_t *src = lb_smem + px * p.stride * p.cu;
-            uint32_t *dst = out + (((size_t)b * p.OH + oh) * p.OW + ow0 + px) * row_words;
+            const int px_off = px * p.stride * p.cu;
+            uint32_t *dstw = out + (((size_t)b * p.OH + oh) * p.OW + ow0 + px) * row_words;
             for (int q = lane; q < row_words; q += 32) {
-                int k = q * 4;
-                int kh = (int)fdiv((uint32_t)k, p.seg), r = k - kh * (int)p.seg.d;
+                const int k = q * 4;
+                int kh = (int)fdiv((uint32_t)k, p.seg), r = k - kh * tap_bytes;
                 uint32_t v = 0;
+                if (r + 4 <= tap_bytes && k + 4 <= p.row_copy) {
+                    const int addr = kh * seg_pitch + px_off + r;
+                    const uint32_t lo = sm_words[addr >> 2], hi = sm_words[(addr >> 2) + 1];
+                    v = __funnelshift_r(lo, hi, (addr & 3) * 8);
+                } else {
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    if (k + e < p.row_copy) v |= (uint32_t)src[kh * seg_bytes + r] << (8 * e);
-                    if (++r == (int)p.seg.d) { r = 0; ++kh; }
+                    for (int e = 0; e < 4; ++e) {
+                        if (k + e < p.row_copy) v |= (uint32_t)lb_smem[kh * seg_pitch + px_off + r] << (8 * e);
+                        if (++r == tap_bytes) { r = 0; ++kh; }
+                    }
                 }
-                dst[q] = v;
+                dstw[q] = v;
             }
         }
     }
@@ -201,7 +225,7 @@ qnn_status im2col_launch(const qnn_conv_desc *d, const void *in, void *lowered, 
     if (mode == 2) {
         // staged variant when the input-row segments of 32 output pixels fit 48 KB
         const int span = (LB_PIX - 1) * d->stride + d->KW;
-        const size_t smem = (size_t)d->KH * span * p.cu;
+        const size_t smem = (size_t)d->KH * ((span * p.cu + 3) & ~3) + 8;   // + one word read past the end
         if (smem <= 48 * 1024 && smem < (1u << 24)) {
             const int chunks = ceil_div(p.OW, LB_PIX);
             long long nb = (long long)d->B * p.OH * chunks;

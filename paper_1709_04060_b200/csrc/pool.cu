@@ -16,23 +16,27 @@ struct PoolParams {
     long long plane_in, plane_out;   // words per bit plane (bit-plane format)
 };
 
+// 16 channels (one uint4) per thread; the padded channel count is a multiple of 16.
 __global__ void __launch_bounds__(256) maxpool_u8_kernel(const PoolParams p) {
-    const long long total = (long long)p.B * p.OH * p.OW * p.cu;
-    const uint32_t *in = reinterpret_cast<const uint32_t *>(p.in);
-    uint32_t *out = reinterpret_cast<uint32_t *>(p.out);
+    const int cu = p.cu >> 2;                                     // 16-byte units per pixel
+    const long long total = (long long)p.B * p.OH * p.OW * cu;
+    const uint4 *in = reinterpret_cast<const uint4 *>(p.in);
+    uint4 *out = reinterpret_cast<uint4 *>(p.out);
     for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
          idx += (long long)gridDim.x * blockDim.x) {
-        const int c = (int)(idx % p.cu);
-        long long t = idx / p.cu;
-        const int ow = (int)(t % p.OW); t /= p.OW;
-        const int oh = (int)(t % p.OH);
-        const int b = (int)(t / p.OH);
-        uint32_t best = 0;
-        for (int i = 0; i < p.k; ++i)
+        const unsigned u = (unsigned)(idx % cu);
+        const unsigned t = (unsigned)(idx / cu);                  // output pixel (< 2^32)
+        const unsigned ow = t % (unsigned)p.OW, t2 = t / (unsigned)p.OW;
+        const unsigned oh = t2 % (unsigned)p.OH, b = t2 / (unsigned)p.OH;
+        uint4 best = make_uint4(0, 0, 0, 0);
+        for (int i = 0; i < p.k; ++i) {
+            const uint4 *row = in + (((size_t)b * p.H + oh * p.stride + i) * p.W + ow * p.stride) * cu + u;
             for (int j = 0; j < p.k; ++j) {
-                const size_t pix = ((size_t)b * p.H + oh * p.stride + i) * p.W + ow * p.stride + j;
-                best = __vmaxu4(best, in[pix * p.cu + c]);
+                const uint4 v = __ldg(row + (size_t)j * cu);
+                best.x = __vmaxu4(best.x, v.x); best.y = __vmaxu4(best.y, v.y);
+                best.z = __vmaxu4(best.z, v.z); best.w = __vmaxu4(best.w, v.w);
             }
+        }
         out[idx] = best;
     }
 }
@@ -79,11 +83,12 @@ qnn_status maxpool_launch(const qnn_pool_desc *d, const void *in, void *out, cud
     p.OH = (d->H - d->k) / d->stride + 1;
     p.OW = (d->W - d->k) / d->stride + 1;
     p.bits = d->bits;
+    if ((long long)d->B * p.OH * p.OW >= 0x7fffffffLL) return QNN_ERR_UNSUPPORTED;
     p.cu = d->fmt == QNN_FMT_INT8 ? round_up(d->C, 16) / 4 : ceil_div(d->C, 32);
     p.plane_in = (long long)d->B * d->H * d->W * p.cu;
     p.plane_out = (long long)d->B * p.OH * p.OW * p.cu;
     const int threads = 256;
-    long long blocks = (p.plane_out + threads - 1) / threads;
+    long long blocks = ((d->fmt == QNN_FMT_INT8 ? p.plane_out / 4 : p.plane_out) + threads - 1) / threads;
     const long long max_blocks = (long long)sm_count() * 16;
     if (blocks > max_blocks) blocks = max_blocks;
     if (d->fmt == QNN_FMT_INT8) {

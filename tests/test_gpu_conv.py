@@ -211,3 +211,31 @@ def test_alexnet_chain_graph_replay(qb):
         assert np.array_equal(logits.cpu().numpy().astype(np.int64), want)
     st, dev = qb.qnn_device_status()
     assert st == 0 and dev == 0
+
+
+@pytest.mark.parametrize("shape", [
+    # B, H, W, C, OC, KH, KW, stride, pad, w_bits, a_bits
+    (2, 9, 10, 5, 20, 3, 3, 1, 1, 8, 8),
+    (1, 7, 7, 3, 17, 3, 3, 2, 1, 8, 8),
+    (3, 12, 11, 6, 33, 5, 4, 1, 2, 4, 4),
+])
+def test_byte_lowering_with_contiguous_pixels_and_padding(qb, shape):
+    """Pixel pitch == C (no per-pixel padding) with zero padding around the image: the
+    staged byte lowering (unaligned-word reads and the byte-by-byte path for words that
+    straddle two filter rows) against the host lowering and the direct convolution."""
+    case = synth.conv_case(970 + shape[3], *shape, w_enc=synth.SIGNED, a_enc=synth.UNSIGNED)
+    x, pitch = device_map(qb, case, INT8, in_pitch=case.C)
+    d = conv_desc(qb, case, INT8, INT8, pitch)
+    npix = case.B * case.OH * case.OW
+    low = torch.full((qb.qnn_conv_lowered_bytes(d),), 0xAB, dtype=torch.uint8, device="cuda")
+    qb.check(qb.qnn_im2col(d, x, low))
+    torch.cuda.synchronize()
+    got = unpack_int8(low.cpu().numpy(), npix, qb.qnn_conv_lowered_k(d), case.a_enc)
+    want = host_im2col(case.In, case.KH, case.KW, case.stride, case.pad, case.C)
+    assert np.array_equal(got, want)
+    Wp = device_weights(qb, case, INT8)
+    out = qb.qconv(d, Wp, x, torch.from_numpy(case.thr).cuda())
+    torch.cuda.synchronize()
+    got = decode_out(out.cpu().numpy(), INT8, case.out_bits, npix, case.OC, False)
+    want = orc.qconv(case.In, case.Wt, case.thr, case.stride, case.pad).reshape(npix, case.OC)
+    assert np.array_equal(got, want)
