@@ -294,12 +294,28 @@ def run_b200(args):
     qdist.finalize()
 
 
-def _time_calls(torch, fn, iters, warmup=3):
-    """Mean device milliseconds of fn(i), CUDA events on the current stream."""
+def _time_calls(torch, fn, iters, warmup=3, graph=False):
+    """Mean device milliseconds of fn(i), CUDA events on the current stream.  With graph=True
+    the `iters` calls are recorded into one CUDA graph and the graph is replayed, which takes
+    the host's per-call cost (a few microseconds of Python and ctypes) out of the number."""
     for i in range(warmup):
         fn(i)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if graph:
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for i in range(iters):
+                fn(i)
+        g.replay()
+        torch.cuda.synchronize()
+        reps = 5
+        e0.record()
+        for _ in range(reps):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / (iters * reps)
     e0.record()
     for i in range(iters):
         fn(warmup + i)
@@ -339,8 +355,9 @@ def run_extras(args):
                 Ap = qb.pack(Ad, bits, c.a_enc, fmt)
                 d = qb.gemm_desc(M, N, K, bits, bits, bits, c.w_enc, c.a_enc, fmt, I8)
                 out = torch.empty(qb.qnn_gemm_out_bytes(d, True), dtype=torch.uint8, device="cuda")
-                ms = _time_calls(torch, lambda i: qb.check(qb.qnn_qgemm(d, Wrot[i % copies], Ap, thr, out)), 4 * copies)
-                ms_warm = _time_calls(torch, lambda i: qb.check(qb.qnn_qgemm(d, Wp, Ap, thr, out)), 50)
+                ms = _time_calls(torch, lambda i: qb.check(qb.qnn_qgemm(d, Wrot[i % copies], Ap, thr, out)),
+                                 4 * copies, graph=True)
+                ms_warm = _time_calls(torch, lambda i: qb.check(qb.qnn_qgemm(d, Wp, Ap, thr, out)), 50, graph=True)
                 alg = Wp.numel() + Ap.numel() + thr.numel() * 4 + N * M
                 skinny.append({"w": bits, "a": bits, "N": N, "fmt": name, "us": 1e3 * ms, "us_l2_warm": 1e3 * ms_warm,
                                "algorithmic_bytes": alg, "gbs": alg / ms / 1e6,
@@ -364,8 +381,9 @@ def run_extras(args):
             thr = torch.from_numpy(c.thr).cuda()
             ws = torch.empty(qb.qnn_conv_workspace_bytes(d), dtype=torch.uint8, device="cuda")
             out = torch.empty(qb.qnn_conv_out_bytes(d, True), dtype=torch.uint8, device="cuda")
-            ms_low = _time_calls(torch, lambda i: qb.check(qb.qnn_im2col(d, x, ws)), 50)
-            ms_all = _time_calls(torch, lambda i: qb.check(qb.qnn_qconv(d, Wp, x, thr, out, ws, ws.numel())), 50)
+            ms_low = _time_calls(torch, lambda i: qb.check(qb.qnn_im2col(d, x, ws)), 50, graph=True)
+            ms_all = _time_calls(torch, lambda i: qb.check(qb.qnn_qconv(d, Wp, x, thr, out, ws, ws.numel())), 50,
+                                 graph=True)
             low_bytes = qb.qnn_conv_lowered_bytes(d) + x.numel()
             conv.append({"B": B, "fmt": name, "im2col_us": 1e3 * ms_low, "im2col_gbs": low_bytes / ms_low / 1e6,
                          "qconv_us": 1e3 * ms_all, "images_per_s": B / ms_all * 1e3,
@@ -386,12 +404,13 @@ def run_extras(args):
                 if kind == "conv":
                     f = lambda i: qb.check(qb.qnn_qconv(d, Wp, x_in, thr, out, plan.workspace, plan.workspace.numel()))
                     per_layer[name + "_lowering"] = round(
-                        1e3 * _time_calls(torch, lambda i: qb.check(qb.qnn_im2col(d, x_in, plan.workspace)), 20), 2)
+                        1e3 * _time_calls(torch, lambda i: qb.check(qb.qnn_im2col(d, x_in, plan.workspace)), 20,
+                                          graph=True), 2)
                 elif kind == "pool":
                     f = lambda i: qb.check(qb.qnn_maxpool(d, x_in, out))
                 else:
                     f = lambda i: qb.check(qb.qnn_qgemm(d, Wp, x_in, thr, out, None, 0))
-                per_layer[name] = round(1e3 * _time_calls(torch, f, 20), 2)
+                per_layer[name] = round(1e3 * _time_calls(torch, f, 20, graph=True), 2)
                 prev = out
             graph, _ = plan.capture(img)
             ms_graph = _time_calls(torch, lambda i: graph.replay(), 30 if B == 1 else 10)
