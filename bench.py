@@ -183,17 +183,39 @@ def run_b200(args):
         problems.append(prob)
     torch.cuda.synchronize()
 
+    # The packer of problem i + 1 (HBM bound) runs on a second stream while the GEMM of
+    # problem i (tensor bound) runs on the main one; events order each GEMM after its packer
+    # and each packer after the GEMM that last read its output buffer.
+    s_pack = torch.cuda.Stream() if args.overlap else None
+
     def step(gemm_events=None, host_io=False):
+        main = torch.cuda.current_stream()
+        if s_pack is not None:
+            s_pack.wait_stream(main)
         for p in problems:
-            if host_io:
-                p["A_log"].copy_(p["A_host"], non_blocking=True)
-            qb.check(qb.qnn_pack(p["pd"], p["A_log"], p["A_packed"]))
+            if s_pack is not None:
+                if "gemm_done" in p:
+                    s_pack.wait_event(p["gemm_done"])
+                with torch.cuda.stream(s_pack):
+                    if host_io:
+                        p["A_log"].copy_(p["A_host"], non_blocking=True)
+                    qb.check(qb.qnn_pack(p["pd"], p["A_log"], p["A_packed"]))
+                    p["packed"] = torch.cuda.Event()
+                    p["packed"].record(s_pack)
+                main.wait_event(p["packed"])
+            else:
+                if host_io:
+                    p["A_log"].copy_(p["A_host"], non_blocking=True)
+                qb.check(qb.qnn_pack(p["pd"], p["A_log"], p["A_packed"]))
             if gemm_events is not None:
                 e0 = torch.cuda.Event(enable_timing=True); e0.record()
             qb.check(qb.qnn_qgemm(p["gd"], p["Wp"], p["A_packed"], p["thr"], p["out"]))
             if gemm_events is not None:
                 e1 = torch.cuda.Event(enable_timing=True); e1.record()
                 gemm_events.append((e0, e1))
+            if s_pack is not None:
+                p["gemm_done"] = torch.cuda.Event()
+                p["gemm_done"].record(main)
             if host_io:
                 p["out_host"].copy_(p["out"], non_blocking=True)
 
@@ -438,6 +460,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--overlap", type=int, default=1,
+                    help="1: activation packer on a second stream, overlapping the previous GEMM (default); 0: one stream")
     ap.add_argument("--workload", default="sweep", choices=["sweep", "extras"],
                     help="sweep: the headline line; extras: the other paper-shaped workloads (one GPU)")
     ap.add_argument("--pairs", default=None,

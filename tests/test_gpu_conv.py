@@ -239,3 +239,35 @@ def test_byte_lowering_with_contiguous_pixels_and_padding(qb, shape):
     got = decode_out(out.cpu().numpy(), INT8, case.out_bits, npix, case.OC, False)
     want = orc.qconv(case.In, case.Wt, case.thr, case.stride, case.pad).reshape(npix, case.OC)
     assert np.array_equal(got, want)
+
+
+def test_config3_conv2_batch64_full(qb):
+    """AlexNet conv2-shaped W1A2 layer at batch 64 (lowered GEMM 256 x 2400 x 46656), the
+    size the benchmark's extras workload times: every output against the direct convolution."""
+    case = synth.conv2_alexnet_case(64)
+    x, pitch = device_map(qb, case, INT8)
+    Wp = device_weights(qb, case, INT8)
+    d = conv_desc(qb, case, INT8, INT8, pitch)
+    out = qb.qconv(d, Wp, x, torch.from_numpy(case.thr).cuda())
+    torch.cuda.synchronize()
+    st, dev = qb.qnn_device_status()
+    assert st == 0 and dev == 0
+    got = decode_out(out.cpu().numpy(), INT8, 2, 64 * 729, 256, False)
+    want = orc.qconv(case.In, case.Wt, case.thr, 1, 2).reshape(64 * 729, 256)
+    assert np.array_equal(got, want)
+
+
+def test_config4_alexnet_batch256_sampled_images(qb):
+    """The chain at batch 256 (the large configuration): images are independent, so the
+    oracle recomputes a sample of them one by one and their logits must match exactly."""
+    from paper_1709_04060_b200.alexnet import AlexNetPlan
+    net = synth.alexnet_case(256)
+    plan = AlexNetPlan(net, 256, "tensor")
+    img = torch.from_numpy(net.image.astype(np.uint8)).cuda()
+    logits = plan.forward(img).cpu().numpy().astype(np.int64)
+    st, dev = qb.qnn_device_status()
+    assert st == 0 and dev == 0
+    for b in (0, 77, 128, 255):
+        one = synth.NetCase(B=1, image=net.image[b:b + 1], weights=net.weights, thr=net.thr)
+        want, _ = onet.forward(one, keep_intermediates=False)
+        assert np.array_equal(logits[b:b + 1], want), f"image {b}"
