@@ -416,7 +416,7 @@ def run_extras(args):
     net_res = []
     for B in (1, 256):
         net = synth.alexnet_case(B)
-        for mode in ("tensor", "bitserial") if B == 1 else ("tensor",):
+        for mode in ("auto", "tensor", "bitserial") if B == 1 else ("auto",):
             plan = AlexNetPlan(net, B, mode)
             img = torch.from_numpy(net.image.astype(np.uint8)).cuda()
             ms = _time_calls(torch, lambda i: plan.forward(img), 30 if B == 1 else 10)

@@ -10,6 +10,11 @@ arithmetic runs in the library's kernels.
   "tensor"     8-bit containers everywhere  (tcgen05 path for every layer)
   "bitserial"  bit planes for the W1A2 layers (bit-serial path; conv1 writes bit
                planes directly from its epilogue, fc7 writes 8-bit codes for fc8)
+  "auto"       per layer, as Section 4.1 of the paper suggests choosing the engine
+               by shape: 8-bit containers (tensor cores) for the convolutions,
+               and, at batch <= 16, bit planes for the fully connected W1A2
+               layers, whose packed weights are streamed once by the few-column
+               bit-serial kernel; at larger batch the same as "tensor"
 """
 import numpy as np
 import torch
@@ -24,8 +29,8 @@ def _round_up(x, m):
 
 
 class AlexNetPlan:
-    def __init__(self, net, B: int, mode: str = "tensor", hw: int = 227):
-        assert mode in ("tensor", "bitserial")
+    def __init__(self, net, B: int, mode: str = "auto", hw: int = 227):
+        assert mode in ("tensor", "bitserial", "auto")
         self.B, self.mode, self.layers = B, mode, list(net.layers)
         self.steps = []          # (kind, desc, tensors...)
         self.names = []
@@ -35,14 +40,17 @@ class AlexNetPlan:
         flat = None
         ws_bytes = 16
         n_layers = len(self.layers)
+        def planes(L):
+            if L.w_bits == 8:
+                return False
+            return mode == "bitserial" or (mode == "auto" and L.kind == "fc" and B <= 16)
+
         for li, L in enumerate(self.layers):
-            eight_bit = L.w_bits == 8
-            want_planes = (mode == "bitserial") and not eight_bit
-            fmt = BITPLANES if want_planes else INT8
+            fmt = BITPLANES if planes(L) else INT8
             assert fmt == fmt_in, "layer input format must match the producer's output format"
             # output format = what the next matrix layer consumes
             nxt = self.layers[li + 1] if li + 1 < n_layers else None
-            out_fmt = BITPLANES if (nxt is not None and mode == "bitserial" and nxt.w_bits != 8) else INT8
+            out_fmt = BITPLANES if (nxt is not None and planes(nxt)) else INT8
             thr = net.thr.get(L.name)
             thr_d = torch.from_numpy(np.ascontiguousarray(thr)).cuda() if thr is not None else None
             Wl = np.asarray(net.weights[L.name])

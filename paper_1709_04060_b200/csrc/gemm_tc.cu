@@ -329,60 +329,69 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams &p, const int *thr
         }
         return;
     }
+    // Eight channels at a time, written so that the threshold loads of all eight are issued
+    // before any of them is used (independent chains interleave instead of running one
+    // after the other).
     uint32_t packed[8];                          // four codes per word, one byte each
     if (OUT_BITS >= 3) {
         // bisection over the channel's sorted thresholds: the row of NT words sits in NT
         // distinct banks, so lanes that look at different slots do not conflict
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            uint32_t w = 0;
+        for (int g = 0; g < 4; ++g) {
+            const int *rows = thr_c + 8 * g * NT;
+            int c[8], t[8];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int j = 4 * k + e, x = acc[j];
-                const int *row = thr_c + j * NT;
-                int c = (x >= row[NT / 2 - 1]) ? NT / 2 : 0;
+            for (int e = 0; e < 8; ++e) t[e] = rows[e * NT + NT / 2 - 1];
 #pragma unroll
-                for (int step = NT / 4; step >= 1; step >>= 1) c += (x >= row[c + step - 1]) ? step : 0;
-                w |= (uint32_t)c << (8 * e);
+            for (int e = 0; e < 8; ++e) c[e] = (acc[8 * g + e] >= t[e]) ? NT / 2 : 0;
+#pragma unroll
+            for (int step = NT / 4; step >= 1; step >>= 1) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) t[e] = rows[e * NT + c[e] + step - 1];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) c[e] += (acc[8 * g + e] >= t[e]) ? step : 0;
             }
-            packed[k] = w;
+            packed[2 * g] = (uint32_t)c[0] | ((uint32_t)c[1] << 8) | ((uint32_t)c[2] << 16) | ((uint32_t)c[3] << 24);
+            packed[2 * g + 1] = (uint32_t)c[4] | ((uint32_t)c[5] << 8) | ((uint32_t)c[6] << 16) | ((uint32_t)c[7] << 24);
         }
     } else if (p.fp_count) {
+        // NT == 4: one float4 of thresholds per channel
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            uint32_t pr[2];
+        for (int g = 0; g < 4; ++g) {
+            float4 t[8];
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int j = 4 * k + 2 * h;
-                const float x0 = __int_as_float(acc[j] + FP_MAGIC_BITS);
-                const float x1 = __int_as_float(acc[j + 1] + FP_MAGIC_BITS);
-                float c = FP_MAGIC;
+            for (int e = 0; e < 8; ++e) t[e] = *reinterpret_cast<const float4 *>(thr_c + (8 * g + e) * NT);
+            uint32_t pr[4];
 #pragma unroll
-                for (int v = 0; v < NT / 4; ++v) {
-                    const float4 t0 = *reinterpret_cast<const float4 *>(thr_c + j * NT + 4 * v);
-                    const float4 t1 = *reinterpret_cast<const float4 *>(thr_c + (j + 1) * NT + 4 * v);
-                    if (4 * v + 0 < N_THR) { c += __saturatef(x0 - t0.x); c = fmaf(__saturatef(x1 - t1.x), 256.f, c); }
-                    if (4 * v + 1 < N_THR) { c += __saturatef(x0 - t0.y); c = fmaf(__saturatef(x1 - t1.y), 256.f, c); }
-                    if (4 * v + 2 < N_THR) { c += __saturatef(x0 - t0.z); c = fmaf(__saturatef(x1 - t1.z), 256.f, c); }
-                    if (4 * v + 3 < N_THR) { c += __saturatef(x0 - t0.w); c = fmaf(__saturatef(x1 - t1.w), 256.f, c); }
+            for (int h = 0; h < 4; ++h) {
+                const float x0 = __int_as_float(acc[8 * g + 2 * h] + FP_MAGIC_BITS);
+                const float x1 = __int_as_float(acc[8 * g + 2 * h + 1] + FP_MAGIC_BITS);
+                const float4 t0 = t[2 * h], t1 = t[2 * h + 1];
+                float s0 = __saturatef(x0 - t0.x), s1 = __saturatef(x1 - t1.x);
+                if (N_THR > 1) {
+                    s0 += __saturatef(x0 - t0.y); s1 += __saturatef(x1 - t1.y);
+                    s0 += __saturatef(x0 - t0.z); s1 += __saturatef(x1 - t1.z);
                 }
-                pr[h] = (uint32_t)__float_as_int(c);
+                pr[h] = (uint32_t)__float_as_int(fmaf(s1, 256.f, s0 + FP_MAGIC));
             }
-            packed[k] = __byte_perm(pr[0], pr[1], 0x5410);
+            packed[2 * g] = __byte_perm(pr[0], pr[1], 0x5410);
+            packed[2 * g + 1] = __byte_perm(pr[2], pr[3], 0x5410);
         }
     } else {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            uint32_t w = 0;
+        for (int g = 0; g < 4; ++g) {
+            int4 t[8];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int j = 4 * k + e;
-                int c = 0;
+            for (int e = 0; e < 8; ++e) t[e] = *reinterpret_cast<const int4 *>(thr_c + (8 * g + e) * NT);
+            int c[8];
 #pragma unroll
-                for (int q = 0; q < N_THR; ++q) c += (acc[j] >= thr_c[j * NT + q]) ? 1 : 0;
-                w |= (uint32_t)c << (8 * e);
+            for (int e = 0; e < 8; ++e) {
+                const int x = acc[8 * g + e];
+                c[e] = (x >= t[e].x) ? 1 : 0;
+                if (N_THR > 1) c[e] += ((x >= t[e].y) ? 1 : 0) + ((x >= t[e].z) ? 1 : 0);
             }
-            packed[k] = w;
+            packed[2 * g] = (uint32_t)c[0] | ((uint32_t)c[1] << 8) | ((uint32_t)c[2] << 16) | ((uint32_t)c[3] << 24);
+            packed[2 * g + 1] = (uint32_t)c[4] | ((uint32_t)c[5] << 8) | ((uint32_t)c[6] << 16) | ((uint32_t)c[7] << 24);
         }
     }
     if (!n_ok) return;

@@ -168,7 +168,7 @@ def test_maxpool(qb, fmt, B, H, C, bits):
     assert np.array_equal(got, want.reshape(-1, C))
 
 
-@pytest.mark.parametrize("mode", ["tensor", "bitserial"])
+@pytest.mark.parametrize("mode", ["tensor", "bitserial", "auto"])
 @pytest.mark.parametrize("B", [1, 3])
 def test_alexnet_chain_per_layer(qb, mode, B):
     """Every intermediate activation tensor and the final logits vs the oracle chain."""
