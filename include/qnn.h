@@ -95,7 +95,9 @@ typedef struct {
     int w_enc, a_enc;     /* qnn_enc                                          */
     int w_fmt, a_fmt;     /* qnn_fmt; both operands must use the same format  */
     int out_fmt;          /* qnn_fmt of the output codes; ignored if thr==NULL*/
-    int path;             /* qnn_path; AUTO selects by operand format         */
+    int path;             /* qnn_path; AUTO selects by operand format, and for a
+                             handful of columns (N <= 16 bit planes, N <= 8
+                             bytes) the one-warp-per-weight-row kernels       */
 } qnn_gemm_desc;
 
 /* Scratch bytes qnn_qgemm needs for this problem (may be 0).  Host only. */

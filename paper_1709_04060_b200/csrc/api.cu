@@ -148,6 +148,10 @@ qnn_status qnn_qgemm(const qnn_gemm_desc *d, const void *W, const void *A, const
     if (!W || !A || !out) return QNN_ERR_INVALID_ARG;
     if (!aligned16(W) || !aligned16(A) || !aligned16(out) || (thr && (reinterpret_cast<uintptr_t>(thr) & 3u)))
         return QNN_ERR_ALIGNMENT;
+    // 8-bit containers with a handful of columns and no path forced: byte dot products,
+    // one warp per weight row (a tensor-core tile would be almost empty)
+    if (d->path == QNN_PATH_AUTO && d->w_fmt == QNN_FMT_INT8 && gemv_i8_fits(d))
+        return gemv_i8_launch(d, W, A, thr, out, (cudaStream_t)stream);
     if (path == QNN_PATH_TCGEN05_I8) return gemm_tc_launch(d, W, A, thr, out, (cudaStream_t)stream);
     // a handful of columns: stream the weight planes once, one warp per row
     if (gemv_planes_fits(d)) return gemv_planes_launch(d, W, A, thr, out, (cudaStream_t)stream);

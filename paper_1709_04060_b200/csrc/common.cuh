@@ -35,6 +35,9 @@ int sm_count();
 qnn_status pack_launch(const qnn_pack_desc *d, const void *logical, void *packed, cudaStream_t s);
 qnn_status gemm_bitserial_launch(const qnn_gemm_desc *d, const void *W, const void *A,
                                  const int32_t *thr, void *out, cudaStream_t s);
+bool gemv_i8_fits(const qnn_gemm_desc *d);
+qnn_status gemv_i8_launch(const qnn_gemm_desc *d, const void *W, const void *A,
+                          const int32_t *thr, void *out, cudaStream_t s);
 bool gemv_planes_fits(const qnn_gemm_desc *d);
 qnn_status gemv_planes_launch(const qnn_gemm_desc *d, const void *W, const void *A,
                               const int32_t *thr, void *out, cudaStream_t s);

@@ -92,6 +92,10 @@ def test_edge_shapes(qb, fmt, M, N, K):
     run_case(qb, case, fmt, INT8, check_pack=True)
     run_case(qb, case, fmt, BITPLANES)
     run_case(qb, case, fmt, INT8, raw=True)
+    if fmt == INT8:            # few columns go to the byte dot-product kernel: also force the tensor cores
+        run_case(qb, case, fmt, INT8, path=2)
+        run_case(qb, case, fmt, BITPLANES, path=2)
+        run_case(qb, case, fmt, INT8, raw=True, path=2)
 
 
 @pytest.mark.parametrize("out_bits", [1, 2, 3, 4])
@@ -108,7 +112,8 @@ def test_eight_bit_layers_tensor_path(qb):
     c1 = synth.gemm_case(500, 96, 3025, 363, 8, 8, synth.SIGNED, synth.UNSIGNED, out_bits=2)
     run_case(qb, c1, INT8, INT8, check_pack=True)
     c8 = synth.gemm_case(501, 1000, 5, 4096, 8, 2, synth.SIGNED, synth.UNSIGNED, out_bits=2)
-    run_case(qb, c8, INT8, INT8, raw=True)
+    run_case(qb, c8, INT8, INT8, raw=True)            # few columns: byte dot-product kernel
+    run_case(qb, c8, INT8, INT8, raw=True, path=2)    # the same on the tensor cores
 
 
 def test_unsorted_thresholds_follow_counting_rule(qb):
@@ -153,9 +158,9 @@ def test_both_tensor_core_kernels(qb, force_tc_kernel, which, M, N, K, w, a):
     every output mode, incl. sizes with ragged M/N/K tails and fewer tiles than SMs."""
     force_tc_kernel(which)
     case = synth.gemm_case(1000 + M + N + K, M, N, K, w, a)
-    run_case(qb, case, INT8, INT8)
-    run_case(qb, case, INT8, BITPLANES)
-    run_case(qb, case, INT8, INT8, raw=True)
+    run_case(qb, case, INT8, INT8, path=2)
+    run_case(qb, case, INT8, BITPLANES, path=2)
+    run_case(qb, case, INT8, INT8, raw=True, path=2)
 
 
 @pytest.mark.parametrize("M,N,K,w,a", [
@@ -265,3 +270,14 @@ def test_config5_square_8192_sampled(qb, bits):
     assert np.array_equal(codes[cols, rows].astype(np.int64), want)
     full_col = orc.qgemm(case.W, case.At[4321:4322], case.thr)[:, 0]
     assert np.array_equal(codes[4321, :].astype(np.int64), full_col)
+
+
+@pytest.mark.parametrize("w_enc,a_enc,w,a", [(1, 0, 8, 8), (1, 1, 4, 8), (0, 0, 3, 2), (0, 1, 2, 4), (2, 0, 1, 2)])
+def test_skinny_byte_kernel_encodings(qb, w_enc, a_enc, w, a):
+    """The few-column kernel on 8-bit containers (4-way byte dot products) with every
+    signedness pair, depths that are not a multiple of 16, ragged M, every output mode."""
+    for K, M, N in ((4100, 333, 3), (1000, 70, 8), (8192, 1000, 1), (33, 5, 7)):
+        case = synth.gemm_case(5300 + K + w, M, N, K, w, a, w_enc, a_enc, out_bits=3)
+        run_case(qb, case, INT8, INT8, check_pack=True)
+        run_case(qb, case, INT8, BITPLANES)
+        run_case(qb, case, INT8, INT8, raw=True)
