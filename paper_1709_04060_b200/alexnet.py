@@ -31,7 +31,7 @@ def _round_up(x, m):
 class AlexNetPlan:
     def __init__(self, net, B: int, mode: str = "auto", hw: int = 227):
         assert mode in ("tensor", "bitserial", "auto")
-        self.B, self.mode, self.layers = B, mode, list(net.layers)
+        self.B, self.mode, self.layers, self.hw = B, mode, list(net.layers), hw
         self.steps = []          # (kind, desc, tensors...)
         self.names = []
         H, C = hw, 3
@@ -136,4 +136,11 @@ class AlexNetPlan:
         return {n: (s[4], s[0], s[1]) for n, s in zip(self.names, self.steps)}
 
     def launches_per_forward(self) -> int:
-        return sum(2 if s[0] == "conv" else 1 for s in self.steps)
+        """Kernels one forward pass launches (counted by the library on a dry call)."""
+        if getattr(self, "_launches", None) is None:
+            img = torch.zeros(self.B, self.hw, self.hw, 3, dtype=torch.uint8, device="cuda")
+            n0 = qb.qnn_launch_count()
+            self.forward(img)
+            torch.cuda.synchronize()
+            self._launches = qb.qnn_launch_count() - n0
+        return self._launches

@@ -1,5 +1,7 @@
 // C ABI entry points: host-side validation, size queries and dispatch.
 // Every step of the path itself runs in the kernels of the sibling files.
+#include <stdlib.h>
+
 #include "common.cuh"
 
 namespace qnn {
@@ -213,6 +215,14 @@ qnn_status qnn_qconv(const qnn_conv_desc *d, const void *Wpacked, const void *in
     if (!workspace || workspace_bytes < qnn_conv_workspace_bytes(d)) return QNN_ERR_WORKSPACE;
     if (!aligned16(Wpacked) || !aligned16(in) || !aligned16(out) || !aligned16(workspace))
         return QNN_ERR_ALIGNMENT;
+    // 8-bit maps on the tensor-core path: the GEMM's loader does the lowering itself (im2col
+    // tensor map) where the shape allows; QNN_CONV_EXPLICIT=1 in the environment keeps the
+    // lowered matrix (measurements, tests)
+    const char *explicit_env = getenv("QNN_CONV_EXPLICIT");
+    if (path == QNN_PATH_TCGEN05_I8 && !(explicit_env && explicit_env[0] == '1')) {
+        st = gemm_tc_conv_launch(d, &g, Wpacked, in, thr, out, (cudaStream_t)stream);
+        if (st != QNN_ERR_UNSUPPORTED) return st;
+    }
     st = im2col_launch(d, in, workspace, (cudaStream_t)stream);
     if (st != QNN_OK) return st;
     return qnn_qgemm(&g, Wpacked, workspace, thr, out, nullptr, 0, stream);

@@ -146,6 +146,17 @@ __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, u
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y) : "memory");
 }
+// im2col-mode load (Section 3.2's lowering done by the copy engine): 128 consecutive output
+// pixels starting at base pixel (w, h, n) of the padded map, filter tap offset (woff, hoff),
+// channels [c, c + 128); pixels outside the image and channels past C read as zero.
+__device__ __forceinline__ void tma_load_im2col(void *dst, const CUtensorMap *map, uint64_t *bar, int c, int w,
+                                                int h, int n, uint16_t woff, uint16_t hoff) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c), "r"(w), "r"(h), "r"(n), "h"(woff), "h"(hoff)
+        : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t ncols) {
@@ -191,6 +202,10 @@ struct TcParams {
     // the depth (k-blocks [0, kb_half) / [kb_half, num_kb)) of tile full_units + r
     int units, full_units, kb_half;
     int share;             // 1: launched as clusters of two CTAs that share the tiles of the last round
+    // Implicit convolution (taps == 0: plain GEMM).  The activation operand is then the
+    // channels-last feature map itself: k-block kb = (filter tap, 128-byte channel chunk), and
+    // the 128 pixels x 128 bytes of a stage are fetched by one im2col-mode TMA load.
+    int taps, cchunks, cv_C, cv_KW, cv_OW, cv_OHW, cv_stride, cv_pad;
 };
 
 // What an epilogue warp needs for the exchange of a shared tile.  The weight ring holds,
@@ -636,13 +651,28 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
             bool ok = true;
             for (int u = blockIdx.x; ok && u < p.units; u += gridDim.x) {
                 const TcUnit un = tc_unit(p, u, BN);
+                int cv_w = 0, cv_h = 0, cv_n = 0;          // base pixel of the unit's first output pixel
+                if (p.taps) {
+                    cv_n = un.p0 / p.cv_OHW;
+                    const int r = un.p0 - cv_n * p.cv_OHW, oh = r / p.cv_OW;
+                    cv_h = oh * p.cv_stride - p.cv_pad;
+                    cv_w = (r - oh * p.cv_OW) * p.cv_stride - p.cv_pad;
+                }
                 for (int kb = un.kb0; kb < un.kb1; ++kb, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1;
                     if (!(ok = mbar_wait(&sm.empty[s], ph ^ 1, abort_flag))) break;
                     mbar_arrive_expect_tx(&sm.full[s], STAGE_BYTES);
-                    tma_load_2d(sm.act[s], &map_act, &sm.full[s], kb * TC_BK, un.p0);
-                    tma_load_2d(sm.wgt[s], &map_wgt, &sm.full[s], kb * TC_BK, un.c0);
+                    if (p.taps) {
+                        const int tap = kb / p.cchunks, cc = kb - tap * p.cchunks;
+                        const int kh = tap / p.cv_KW, kw = tap - kh * p.cv_KW;
+                        tma_load_im2col(sm.act[s], &map_act, &sm.full[s], cc * TC_BK, cv_w, cv_h, cv_n,
+                                        (uint16_t)kw, (uint16_t)kh);
+                        tma_load_2d(sm.wgt[s], &map_wgt, &sm.full[s], tap * p.cv_C + cc * TC_BK, un.c0);
+                    } else {
+                        tma_load_2d(sm.act[s], &map_act, &sm.full[s], kb * TC_BK, un.p0);
+                        tma_load_2d(sm.wgt[s], &map_wgt, &sm.full[s], kb * TC_BK, un.c0);
+                    }
                 }
             }
             if (!ok) {
@@ -672,9 +702,15 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
                     if (kb == un.kb0) QNN_TRACE(6, tcount);
                     const uint64_t da = umma_smem_desc(smem_u32(sm.act[s]));
                     const uint64_t db = umma_smem_desc(smem_u32(sm.wgt[s]));
+                    // a channel chunk may hold fewer than 128 real bytes: skip the all-zero MMAs
+                    int nk = TC_BK / 32;
+                    if (p.taps) {
+                        const int left = p.cv_C - (kb % p.cchunks) * TC_BK;
+                        if (left < TC_BK) nk = (left + 31) >> 5;
+                    }
 #pragma unroll
                     for (int kk = 0; kk < TC_BK / 32; ++kk)   // 32 depth bytes per MMA: +2 in 16-byte units
-                        umma_i8(d_tmem, da + 2 * kk, db + 2 * kk, p.idesc, (kb > un.kb0) || kk != 0);
+                        if (kk < nk) umma_i8(d_tmem, da + 2 * kk, db + 2 * kk, p.idesc, (kb > un.kb0) || kk != 0);
                     umma_commit(&sm.empty[s]);
                 }
                 if (ok) umma_commit(&sm.tmem_full[buf]);
@@ -920,6 +956,39 @@ static bool make_map(CUtensorMap *map, const void *base, int rows, int K, int ld
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+typedef CUresult (*EncodeIm2colFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const int *, const int *, cuuint32_t, cuuint32_t,
+                                   const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeIm2colFn encode_im2col_fn() {
+    static EncodeIm2colFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeIm2colFn)p;
+    }
+    return fn;
+}
+
+// Channels-last byte map [B][H][W][pitch] seen through an im2col tensor map: a load yields 128
+// pixels x 128 channel bytes; base pixels range over the padded map so that every filter tap
+// (offset 0 .. K-1 from the base) of every output pixel is addressable, out of range = 0.
+static bool make_im2col_map(CUtensorMap *map, const void *base, const qnn_conv_desc *d, int pitch) {
+    EncodeIm2colFn fn = encode_im2col_fn();
+    if (!fn) return false;
+    cuuint64_t dims[4] = {(cuuint64_t)d->C, (cuuint64_t)d->W, (cuuint64_t)d->H, (cuuint64_t)d->B};
+    cuuint64_t strides[3] = {(cuuint64_t)pitch, (cuuint64_t)pitch * d->W, (cuuint64_t)pitch * d->W * d->H};
+    int lower[2] = {-d->pad, -d->pad};
+    int upper[2] = {d->pad - (d->KW - 1), d->pad - (d->KH - 1)};
+    cuuint32_t estr[4] = {1, (cuuint32_t)d->stride, (cuuint32_t)d->stride, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(base), dims, strides, lower, upper,
+              (cuuint32_t)TC_BK, (cuuint32_t)TC_BP, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int BN, int STAGES, int OUT_MODE, int OUT_BITS>
 static qnn_status launch_cfg(const CUtensorMap &ma, const CUtensorMap &mw, const TcParams &p, cudaStream_t s) {
     auto kern = qgemm_tc_kernel<BN, STAGES, OUT_MODE, OUT_BITS>;
@@ -1025,17 +1094,25 @@ static bool tc_plan(const qnn_gemm_desc *d, int sms, TcPlan *pl) {
     return true;
 }
 
-qnn_status gemm_tc_launch(const qnn_gemm_desc *d, const void *W, const void *A, const int32_t *thr,
-                          void *out, cudaStream_t s) {
+// cv != nullptr: implicit convolution, A is the feature map (see TcParams); d is the lowered GEMM.
+static qnn_status tc_launch(const qnn_gemm_desc *d, const qnn_conv_desc *cv, const void *W, const void *A,
+                            const int32_t *thr, void *out, cudaStream_t s) {
     const int ld = round_up(d->K, 16);
     const int sms = sm_count();
-    const bool pair = choose_pair_kernel(d, sms);
+    const bool pair = !cv && choose_pair_kernel(d, sms);
 
     TcParams p;
     p.thr = thr; p.out = out; p.M = d->M; p.N = d->N; p.K = d->K;
     p.num_kb = ceil_div(d->K, TC_BK);
     p.ld_out = round_up(d->M, 16);
     p.kb_half = 0; p.share = 0;
+    p.taps = 0; p.cchunks = 1; p.cv_C = p.cv_KW = p.cv_OW = p.cv_OHW = p.cv_stride = 1; p.cv_pad = 0;
+    if (cv) {
+        p.taps = cv->KH * cv->KW; p.cchunks = ceil_div(cv->C, TC_BK);
+        p.cv_C = cv->C; p.cv_KW = cv->KW; p.cv_stride = cv->stride; p.cv_pad = cv->pad;
+        p.cv_OW = qnn_conv_out_w(cv); p.cv_OHW = qnn_conv_out_h(cv) * p.cv_OW;
+        p.num_kb = p.taps * p.cchunks;
+    }
     const double wmax = d->w_enc == QNN_ENC_BIPOLAR ? 1.0
                         : (d->w_enc == QNN_ENC_SIGNED ? double(1 << (d->w_bits - 1)) : double((1 << d->w_bits) - 1));
     const double amax = d->a_enc == QNN_ENC_BIPOLAR ? 1.0
@@ -1069,12 +1146,45 @@ qnn_status gemm_tc_launch(const qnn_gemm_desc *d, const void *W, const void *A, 
         p.kb_half = (p.num_kb + 1) / 2;
     }
     p.idesc = idesc_base | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(TC_BP >> 4) << 24);
-    if (!make_map(&ma, A, d->N, d->K, ld, TC_BP) || !make_map(&mw, W, d->M, d->K, ld, bn)) return QNN_ERR_CUDA;
+    if (cv) {
+        const int pitch = cv->in_pitch ? cv->in_pitch : round_up(cv->C, 16);
+        if (!make_im2col_map(&ma, A, cv, pitch)) return QNN_ERR_UNSUPPORTED;     // caller lowers explicitly
+    } else if (!make_map(&ma, A, d->N, d->K, ld, TC_BP)) {
+        return QNN_ERR_CUDA;
+    }
+    if (!make_map(&mw, W, d->M, d->K, ld, bn)) return QNN_ERR_CUDA;
     switch (bn) {
         case 256: return launch_out<256, 4>(mode, d->out_bits, ma, mw, p, s);
         case 128: return launch_out<128, 6>(mode, d->out_bits, ma, mw, p, s);
         default:  return launch_out<32, 8>(mode, d->out_bits, ma, mw, p, s);
     }
+}
+
+qnn_status gemm_tc_launch(const qnn_gemm_desc *d, const void *W, const void *A, const int32_t *thr,
+                          void *out, cudaStream_t s) {
+    return tc_launch(d, nullptr, W, A, thr, out, s);
+}
+
+// Convolution without a lowered matrix: the GEMM's loader reads the 8-bit channels-last map
+// through an im2col tensor map.  UNSUPPORTED when the shape needs the explicit lowering
+// (channel count or pixel pitch not a multiple of 16, stride other than 1).
+qnn_status gemm_tc_conv_launch(const qnn_conv_desc *cv, const qnn_gemm_desc *g, const void *W, const void *in,
+                               const int32_t *thr, void *out, cudaStream_t s) {
+    const int pitch = cv->in_pitch ? cv->in_pitch : round_up(cv->C, 16);
+    if (cv->fmt != QNN_FMT_INT8 || (cv->C % 16) != 0 || (pitch % 16) != 0 || cv->stride != 1)
+        return QNN_ERR_UNSUPPORTED;
+    if (cv->KH > 255 || cv->KW > 255) return QNN_ERR_UNSUPPORTED;
+    // A single round of tiles is bound by the latency of its serial depth loop.  When the channel
+    // count is not a multiple of 128 that loop has more (partly empty) k-blocks here than over the
+    // dense lowered matrix, so small problems keep the explicit lowering.
+    TcPlan pl;
+    if (!tc_plan(g, sm_count(), &pl)) return QNN_ERR_UNSUPPORTED;
+    const long long tiles = (long long)pl.tiles_p * pl.tiles_c;
+    const char *force = getenv("QNN_CONV_IMPLICIT");          // "1": skip this heuristic (tests)
+    if (!(force && force[0] == '1') && tiles <= sm_count() &&
+        cv->KH * cv->KW * ceil_div(cv->C, TC_BK) > ceil_div(g->K, TC_BK))
+        return QNN_ERR_UNSUPPORTED;
+    return tc_launch(g, cv, W, in, thr, out, s);
 }
 
 #ifdef QNN_TC_TRACE

@@ -94,10 +94,19 @@ def test_im2col_matches_host_lowering(qb, fmt, shape):
     assert np.array_equal(got, want)
 
 
+@pytest.mark.parametrize("lowering", ["auto", "explicit"])
 @pytest.mark.parametrize("fmt", [BITPLANES, INT8])
 @pytest.mark.parametrize("out_fmt", [BITPLANES, INT8])
 @pytest.mark.parametrize("shape", CONV_CASES)
-def test_qconv_matches_direct_convolution(qb, fmt, out_fmt, shape):
+def test_qconv_matches_direct_convolution(qb, monkeypatch, lowering, fmt, out_fmt, shape):
+    """auto: 8-bit maps with C a multiple of 16 and stride 1 are lowered inside the GEMM's
+    loader (im2col tensor map); explicit: always through the lowered matrix."""
+    if lowering == "explicit":
+        if fmt == BITPLANES:
+            pytest.skip("bit-plane maps are always lowered explicitly")
+        monkeypatch.setenv("QNN_CONV_EXPLICIT", "1")
+    else:
+        monkeypatch.setenv("QNN_CONV_IMPLICIT", "1")
     case = synth.conv_case(900 + shape[4], *shape)
     x, pitch = device_map(qb, case, fmt)
     Wp = device_weights(qb, case, fmt)
@@ -271,3 +280,41 @@ def test_config4_alexnet_batch256_sampled_images(qb):
         one = synth.NetCase(B=1, image=net.image[b:b + 1], weights=net.weights, thr=net.thr)
         want, _ = onet.forward(one, keep_intermediates=False)
         assert np.array_equal(logits[b:b + 1], want), f"image {b}"
+
+
+@pytest.mark.parametrize("shape", [
+    # B, H, W, C, OC, KH, KW, stride, pad, w_bits, a_bits
+    (3, 13, 13, 384, 256, 3, 3, 1, 1, 1, 2),      # conv5 shape: three 128-byte channel chunks per tap
+    (2, 27, 27, 96, 256, 5, 5, 1, 2, 1, 2),       # conv2 shape: a 96-byte chunk (three of four MMAs)
+    (5, 6, 7, 48, 40, 3, 2, 1, 0, 2, 2),          # no padding, ragged everything
+    (1, 5, 5, 272, 33, 5, 5, 1, 4, 3, 3),         # padding larger than half the filter, 128+128+16 bytes
+    (200, 4, 4, 16, 70, 2, 2, 1, 1, 4, 4),        # many small images: tiles span several images
+])
+def test_implicit_convolution_shapes(qb, monkeypatch, shape):
+    """Convolution with the lowering done by the tensor-core kernel's loader, against the direct
+    convolution; the explicit-lowering path must give the same bytes."""
+    monkeypatch.setenv("QNN_CONV_IMPLICIT", "1")      # also where the library would rather lower explicitly
+    case = synth.conv_case(990 + shape[3], *shape)
+    x, pitch = device_map(qb, case, INT8)
+    Wp = device_weights(qb, case, INT8)
+    npix = case.B * case.OH * case.OW
+    thr = torch.from_numpy(case.thr).cuda()
+    for out_fmt in (INT8, BITPLANES):
+        d = conv_desc(qb, case, INT8, out_fmt, pitch)
+        out = qb.qconv(d, Wp, x, thr)
+        torch.cuda.synchronize()
+        st, dev = qb.qnn_device_status()
+        assert st == 0 and dev == 0
+        got = decode_out(out.cpu().numpy(), out_fmt, case.out_bits, npix, case.OC, False)
+        want = orc.qconv(case.In, case.Wt, case.thr, case.stride, case.pad).reshape(npix, case.OC)
+        assert np.array_equal(got, want)
+    d = conv_desc(qb, case, INT8, INT8, pitch)
+    n0 = qb.qnn_launch_count()
+    raw = qb.qconv(d, Wp, x, None).clone()
+    assert qb.qnn_launch_count() - n0 == 1            # one fused kernel, no lowering kernel
+    monkeypatch.setenv("QNN_CONV_EXPLICIT", "1")
+    n0 = qb.qnn_launch_count()
+    raw_explicit = qb.qconv(d, Wp, x, None)
+    assert qb.qnn_launch_count() - n0 == 2            # lowering + GEMM
+    torch.cuda.synchronize()
+    assert torch.equal(raw, raw_explicit)
