@@ -140,10 +140,12 @@ typedef struct {
 int qnn_conv_out_h(const qnn_conv_desc *d);
 int qnn_conv_out_w(const qnn_conv_desc *d);
 
-/* Depth of the lowered GEMM: BITPLANES -> 32 * KH*KW*ceil(C/32) (each pixel is
- * padded to whole words, Section 3.2); INT8 -> KH*KW*C.  The weight operand
- * passed to qnn_qconv must be packed with this K and the same per-pixel
- * padding: logical weight row = (kh, kw, c) with c fastest.  Host only. */
+/* Depth of the lowered GEMM.  BITPLANES: 32 * KH*KW*ceil(C/32) (each pixel is
+ * padded to whole words, Section 3.2).  INT8: KH*KW*C when C is a multiple of
+ * 16; otherwise KH * (KW*C rounded up to 16): the KW*C bytes of each filter row
+ * form one run, zero padded to a 16-byte boundary.  The weight operand passed
+ * to qnn_qconv must be packed with this K and the same padding (zeros):
+ * logical weight row = (kh, kw, c) with c fastest.  Host only. */
 int qnn_conv_lowered_k(const qnn_conv_desc *d);
 
 /* Bytes of the lowered matrix / of qnn_qconv's workspace.  Host only. */
@@ -158,8 +160,8 @@ size_t qnn_conv_out_bytes(const qnn_conv_desc *d, int has_thresholds);
  *   fmt BITPLANES: in uint32 [a_bits][B][H][W][ceil(C/32)]
  *                  -> lowered uint32 [a_bits][B*OH*OW][KH*KW*ceil(C/32)]
  *   fmt INT8:      in uint8 [B][H][W][in_pitch] (the first C bytes of a pixel
- *                  are its channels) -> lowered uint8 [B*OH*OW][ld],
- *                  ld = KH*KW*C rounded up to 16, pad bytes zero.
+ *                  are its channels; in_pitch a multiple of 16 when C is)
+ *                  -> lowered uint8 [B*OH*OW][qnn_conv_lowered_k], pad bytes zero.
  * The lowered matrix is the activation operand A of qnn_qgemm (N = B*OH*OW). */
 qnn_status qnn_im2col(const qnn_conv_desc *d, const void *in, void *lowered, void *stream);
 

@@ -58,14 +58,7 @@ class AlexNetPlan:
                 d = qb.qnn_conv_desc(B, H, H, C, in_pitch if fmt == INT8 else 0, L.OC, L.KH, L.KW,
                                      L.stride, L.pad, L.w_bits, L.a_bits, max(L.out_bits, 1),
                                      L.w_enc, qb.QNN_ENC_UNSIGNED, fmt, out_fmt, qb.QNN_PATH_AUTO)
-                K = qb.qnn_conv_lowered_k(d)
-                if fmt == BITPLANES:
-                    cw = (C + 31) // 32
-                    Wpad = np.zeros((L.OC, L.KH * L.KW, cw * 32), dtype=Wl.dtype)
-                    Wpad[:, :, :C] = Wl.reshape(L.OC, L.KH * L.KW, C)
-                    Wflat = Wpad.reshape(L.OC, K)
-                else:
-                    Wflat = Wl.reshape(L.OC, K)
+                Wflat = qb.conv_weight_rows(d, Wl)
                 Wp = qb.pack(qb.to_device_logical(Wflat, L.w_enc), L.w_bits, L.w_enc, fmt)
                 out = torch.empty(qb.qnn_conv_out_bytes(d, thr is not None), dtype=torch.uint8, device="cuda")
                 ws_bytes = max(ws_bytes, qb.qnn_conv_workspace_bytes(d))

@@ -270,6 +270,25 @@ def qgemm(d: qnn_gemm_desc, W, A, thr, out=None, stream=None) -> torch.Tensor:
     return out
 
 
+def conv_weight_rows(d: qnn_conv_desc, Wt):
+    """Logical filters [OC][KH][KW][C] (numpy) laid out as the rows [OC][qnn_conv_lowered_k]
+    that `pack` expects for this convolution: per-pixel padding to 32 channels for bit planes,
+    per-filter-row padding to 16 bytes for 8-bit maps whose C is not a multiple of 16."""
+    import numpy as np
+    OC, KH, KW, C = Wt.shape
+    K = qnn_conv_lowered_k(d)
+    if d.fmt == QNN_FMT_BITPLANES:
+        cp = (C + 31) // 32 * 32
+        rows = np.zeros((OC, KH * KW, cp), dtype=Wt.dtype)
+        rows[:, :, :C] = Wt.reshape(OC, KH * KW, C)
+    elif C % 16 == 0:
+        rows = Wt
+    else:
+        rows = np.zeros((OC, KH, K // KH), dtype=Wt.dtype)
+        rows[:, :, :KW * C] = Wt.reshape(OC, KH, KW * C)
+    return np.ascontiguousarray(rows.reshape(OC, K))
+
+
 def qconv(d: qnn_conv_desc, Wpacked, inp, thr, out=None, workspace=None, stream=None) -> torch.Tensor:
     if out is None:
         out = _dev_bytes(qnn_conv_out_bytes(d, thr is not None))

@@ -170,7 +170,8 @@ int qnn_conv_out_w(const qnn_conv_desc *d) {
 int qnn_conv_lowered_k(const qnn_conv_desc *d) {
     if (!d) return 0;
     if (d->fmt == QNN_FMT_BITPLANES) return 32 * d->KH * d->KW * ceil_div(d->C, 32);
-    return d->KH * d->KW * d->C;
+    if (d->C % 16 == 0) return d->KH * d->KW * d->C;
+    return d->KH * round_up(d->KW * d->C, 16);       // one zero-padded run per filter row
 }
 
 size_t qnn_conv_lowered_bytes(const qnn_conv_desc *d) {

@@ -2,8 +2,8 @@
 // bit position per plane, every pixel padded to whole words, so lowering moves
 // whole words -- one im2col per activation bit plane, no masking or shifting.
 // The same kernel lowers 8-bit-container maps in 16-byte units (channel count a
-// multiple of 16); a byte-granular variant covers other channel counts (the
-// 3-channel input image of the first layer).
+// multiple of 16); other channel counts (the 3-channel input image of the first
+// layer) are lowered as one zero-padded run of bytes per filter row.
 //
 // One warp per output pixel: the pixel's coordinates are decoded once, lanes
 // stream the lowered row (kh, kw, c order, c fastest) with coalesced stores.
@@ -74,63 +74,32 @@ __global__ void __launch_bounds__(256) lower_units_kernel(const LowerParams p) {
     }
 }
 
-// Byte-granular lowering of 8-bit maps: a thread assembles 4 consecutive output bytes.
-__global__ void __launch_bounds__(256) lower_bytes_kernel(const LowerParams p) {
-    const int lane = threadIdx.x & 31;
-    const long long warp0 = (blockIdx.x * (long long)blockDim.x + threadIdx.x) >> 5;
-    const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
-    const uint8_t *in = reinterpret_cast<const uint8_t *>(p.in);
-    uint32_t *out = reinterpret_cast<uint32_t *>(p.out);
-    const int row_words = p.row_units >> 2;        // row pitch is a multiple of 16 bytes
-    for (long long pix = warp0; pix < p.npix; pix += nwarps) {
-        const int b = (int)(pix / (p.OH * p.OW));
-        const uint32_t rem = (uint32_t)(pix - (long long)b * p.OH * p.OW);
-        const int oh = (int)fdiv(rem, p.owd), ow = (int)(rem - oh * p.OW);
-        const int ih0 = oh * p.stride - p.pad, iw0 = ow * p.stride - p.pad;
-        const uint8_t *src = in + (size_t)b * p.H * p.W * p.pitch;
-        uint32_t *dst = out + (size_t)pix * row_words;
-        for (int q = lane; q < row_words; q += 32) {
-            int k = q * 4;
-            int kh = (int)fdiv(k, p.seg), r = k - kh * (int)p.seg.d;
-            int kw = (int)fdiv(r, p.cud), c = r - kw * p.cu;
-            uint32_t v = 0;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                if (k + e < p.row_copy) {
-                    const int ih = ih0 + kh, iw = iw0 + kw;
-                    if (ih >= 0 && ih < p.H && iw >= 0 && iw < p.W)
-                        v |= (uint32_t)src[((size_t)ih * p.W + iw) * p.pitch + c] << (8 * e);
-                }
-                if (++c == p.cu) { c = 0; if (++kw == p.KW) { kw = 0; ++kh; } }
-            }
-            dst[q] = v;
-        }
-    }
-}
+// Lowering of 8-bit maps whose channel count is not a multiple of 16 (the 3-channel input
+// image of the first layer).  The lowered row keeps one run per filter row: the KW*C bytes that
+// row contributes, zero padded to a multiple of 16, so every run starts on a 16-byte boundary
+// of the output (the weight rows carry the same padding).  A CTA takes up to LR_PIX consecutive
+// output pixels of one output row, stages the KH input-row segments they touch in shared memory
+// (compact, C bytes per pixel, zeros outside the image), then one thread per (pixel, filter
+// row) turns its run -- contiguous in the staged segment -- into 16-byte stores: an unaligned
+// 16-byte read is five aligned words and four funnel shifts.
+constexpr int LR_PIX = 64;
 
-// Byte-granular lowering through shared memory: a CTA takes LB_PIX consecutive output
-// pixels of one output row, stages the KH input-row segments they touch (compact, C bytes
-// per pixel, zeros outside the image) and then assembles the lowered rows from shared
-// memory, one warp per output pixel, 4 bytes per lane and step, with coalesced stores.
-constexpr int LB_PIX = 32;
-
-__global__ void __launch_bounds__(256) lower_bytes_smem_kernel(const LowerParams p, int chunks, int span) {
-    extern __shared__ __align__(16) uint8_t lb_smem[];   // [KH][seg_pitch], seg_pitch = span * C rounded up to 4
+__global__ void __launch_bounds__(256) lower_runs_kernel(const LowerParams p, int chunks, int span, int run,
+                                                         int runp) {
+    extern __shared__ __align__(16) uint8_t lr_smem[];   // [KH][seg_pitch] + slack
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint8_t *in = reinterpret_cast<const uint8_t *>(p.in);
-    uint32_t *out = reinterpret_cast<uint32_t *>(p.out);
-    const uint32_t *sm_words = reinterpret_cast<const uint32_t *>(lb_smem);
-    const int row_words = p.row_units >> 2;
+    const uint32_t *sm_words = reinterpret_cast<const uint32_t *>(lr_smem);
     const int seg_bytes = span * p.cu;                   // bytes of one staged input-row segment
     const int seg_pitch = (seg_bytes + 3) & ~3;
-    const int tap_bytes = (int)p.seg.d;                  // KW * C: bytes one filter row contributes
+    const int vecs = runp >> 4;                          // 16-byte stores per run
     const long long jobs = (long long)p.B * p.OH * chunks;
     for (long long job = blockIdx.x; job < jobs; job += gridDim.x) {
         const int chunk = (int)(job % chunks);
         const long long t = job / chunks;
         const int oh = (int)(t % p.OH), b = (int)(t / p.OH);
-        const int ow0 = chunk * LB_PIX;
-        const int npx = min(LB_PIX, p.OW - ow0);
+        const int ow0 = chunk * LR_PIX;
+        const int npx = min(LR_PIX, p.OW - ow0);
         const int ih0 = oh * p.stride - p.pad, iw0 = ow0 * p.stride - p.pad;
         __syncthreads();                                 // previous job's readers are done
         // stage: one warp per filter row, lanes along the bytes of the segment
@@ -138,7 +107,7 @@ __global__ void __launch_bounds__(256) lower_bytes_smem_kernel(const LowerParams
             const int ih = ih0 + kh;
             const bool row_ok = ih >= 0 && ih < p.H;
             const uint8_t *row = in + (((size_t)b * p.H + (row_ok ? ih : 0)) * p.W) * p.pitch;
-            uint8_t *dst = lb_smem + kh * seg_pitch;
+            uint8_t *dst = lr_smem + kh * seg_pitch;
             if (p.pitch == p.cu) {
                 // pixels are contiguous: byte r of the segment is byte iw0*C + r of the image row
                 const int lo = max(0, -iw0) * p.cu, hi = min(span, p.W - iw0) * p.cu;
@@ -155,28 +124,27 @@ __global__ void __launch_bounds__(256) lower_bytes_smem_kernel(const LowerParams
             }
         }
         __syncthreads();
-        // assemble: within one filter row the bytes of a lowered row are contiguous in the
-        // staged segment, so a word is an unaligned 4-byte read (two aligned words and a
-        // funnel shift) unless it straddles two filter rows
-        for (int px = warp; px < npx; px += 8) {
-            const int px_off = px * p.stride * p.cu;
-            uint32_t *dstw = out + (((size_t)b * p.OH + oh) * p.OW + ow0 + px) * row_words;
-            for (int q = lane; q < row_words; q += 32) {
-                const int k = q * 4;
-                int kh = (int)fdiv((uint32_t)k, p.seg), r = k - kh * tap_bytes;
-                uint32_t v = 0;
-                if (r + 4 <= tap_bytes && k + 4 <= p.row_copy) {
-                    const int addr = kh * seg_pitch + px_off + r;
-                    const uint32_t lo = sm_words[addr >> 2], hi = sm_words[(addr >> 2) + 1];
-                    v = __funnelshift_r(lo, hi, (addr & 3) * 8);
-                } else {
+        uint4 *out_row = reinterpret_cast<uint4 *>(p.out) +
+                         (((size_t)b * p.OH + oh) * p.OW + ow0) * (size_t)(p.KH * vecs);
+        for (int task = threadIdx.x; task < npx * p.KH; task += blockDim.x) {
+            const int px = (int)fdiv((uint32_t)task, p.seg), kh = task - px * p.KH;    // p.seg divides by KH here
+            const int src = kh * seg_pitch + px * p.stride * p.cu;
+            const int sh = (src & 3) * 8;
+            const uint32_t *w = sm_words + (src >> 2);
+            uint4 *dst = out_row + (size_t)task * vecs;
+            for (int v = 0; v < vecs; ++v) {
+                uint32_t x[5];
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        if (k + e < p.row_copy) v |= (uint32_t)lb_smem[kh * seg_pitch + px_off + r] << (8 * e);
-                        if (++r == tap_bytes) { r = 0; ++kh; }
-                    }
+                for (int i = 0; i < 5; ++i) x[i] = w[4 * v + i];
+                uint32_t o[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    o[i] = __funnelshift_r(x[i], x[i + 1], sh);
+                    const int valid = run - (16 * v + 4 * i);          // bytes of this word inside the run
+                    if (valid <= 0) o[i] = 0;
+                    else if (valid < 4) o[i] &= (1u << (8 * valid)) - 1u;
                 }
-                dstw[q] = v;
+                dst[v] = make_uint4(o[0], o[1], o[2], o[3]);
             }
         }
     }
@@ -195,7 +163,8 @@ qnn_status im2col_launch(const qnn_conv_desc *d, const void *in, void *lowered, 
     const int threads = 256;
     const long long max_blocks = (long long)sm_count() * 16;
 
-    int mode;   // 0 words, 1 16-byte units, 2 bytes
+    int mode;   // 0 words, 1 16-byte units, 2 padded runs of bytes
+    int run = 0, runp = 0;
     if (d->fmt == QNN_FMT_BITPLANES) {
         mode = 0;
         p.planes = d->a_bits;
@@ -203,41 +172,42 @@ qnn_status im2col_launch(const qnn_conv_desc *d, const void *in, void *lowered, 
         p.row_copy = d->KH * d->KW * p.cu; p.row_units = p.row_copy;
     } else {
         const int pitch = d->in_pitch ? d->in_pitch : round_up(d->C, 16);
-        const int ld = round_up(d->KH * d->KW * d->C, 16);
         p.planes = 1;
         if (d->C % 16 == 0 && pitch % 16 == 0) {
             mode = 1;
             p.cu = d->C / 16; p.pitch = pitch / 16;
-            p.row_copy = d->KH * d->KW * p.cu; p.row_units = ld / 16;
+            p.row_copy = d->KH * d->KW * p.cu; p.row_units = p.row_copy;
+        } else if (d->C % 16 == 0) {
+            return QNN_ERR_ALIGNMENT;            // 16-byte channel groups need a 16-byte pixel pitch
         } else {
             mode = 2;
             p.cu = d->C; p.pitch = pitch;
-            p.row_copy = d->KH * d->KW * d->C; p.row_units = ld;
+            run = d->KW * d->C; runp = round_up(run, 16);
+            p.row_copy = d->KH * runp; p.row_units = p.row_copy;
         }
     }
-    if (p.row_units >= 65536 || d->KW * p.cu >= 65536) return QNN_ERR_UNSUPPORTED;
-    p.seg = make_fastdiv(d->KW * p.cu);
+    if (p.row_units >= 65536 * 16 || d->KW * p.cu >= 65536) return QNN_ERR_UNSUPPORTED;
     p.cud = make_fastdiv(p.cu);
 
+    if (mode == 2) {
+        const int span = (LR_PIX - 1) * d->stride + d->KW;
+        const size_t smem = (size_t)d->KH * ((span * p.cu + 3) & ~3) + 32;      // slack: reads run past a segment
+        if (smem > 48 * 1024 || LR_PIX * d->KH >= 65536) return QNN_ERR_UNSUPPORTED;
+        p.seg = make_fastdiv(d->KH);
+        const int chunks = ceil_div(p.OW, LR_PIX);
+        long long nb = (long long)d->B * p.OH * chunks;
+        if (nb > max_blocks) nb = max_blocks;
+        lower_runs_kernel<<<(unsigned)nb, threads, smem, s>>>(p, chunks, span, run, runp);
+        count_launch();
+        return launch_status();
+    }
+    if (p.row_units >= 65536) return QNN_ERR_UNSUPPORTED;
+    p.seg = make_fastdiv(d->KW * p.cu);
     const long long jobs = p.npix * p.planes;
     long long blocks = (jobs * 32 + threads - 1) / threads;
     if (blocks > max_blocks) blocks = max_blocks;
-    if (mode == 2) {
-        // staged variant when the input-row segments of 32 output pixels fit 48 KB
-        const int span = (LB_PIX - 1) * d->stride + d->KW;
-        const size_t smem = (size_t)d->KH * ((span * p.cu + 3) & ~3) + 8;   // + one word read past the end
-        if (smem <= 48 * 1024 && smem < (1u << 24)) {
-            const int chunks = ceil_div(p.OW, LB_PIX);
-            long long nb = (long long)d->B * p.OH * chunks;
-            if (nb > max_blocks) nb = max_blocks;
-            lower_bytes_smem_kernel<<<(unsigned)nb, threads, smem, s>>>(p, chunks, span);
-            count_launch();
-            return launch_status();
-        }
-    }
     if (mode == 0) lower_units_kernel<uint32_t><<<(unsigned)blocks, threads, 0, s>>>(p);
-    else if (mode == 1) lower_units_kernel<uint4><<<(unsigned)blocks, threads, 0, s>>>(p);
-    else lower_bytes_kernel<<<(unsigned)blocks, threads, 0, s>>>(p);
+    else lower_units_kernel<uint4><<<(unsigned)blocks, threads, 0, s>>>(p);
     count_launch();
     return launch_status();
 }

@@ -20,8 +20,9 @@ def qb():
     return binding
 
 
-def host_im2col(In, KH, KW, stride, pad, c_pad):
-    """Test-side lowering: rows (b, oh, ow), columns (kh, kw, c) with each pixel padded to c_pad."""
+def host_im2col(In, KH, KW, stride, pad, c_pad, run_pad=False):
+    """Test-side lowering: rows (b, oh, ow), columns (kh, kw, c) with each pixel padded to c_pad;
+    run_pad: every filter row's KW*c_pad values are zero padded to a multiple of 16."""
     B, H, Wd, C = In.shape
     OH = (H + 2 * pad - KH) // stride + 1
     OW = (Wd + 2 * pad - KW) // stride + 1
@@ -31,6 +32,10 @@ def host_im2col(In, KH, KW, stride, pad, c_pad):
     for oh in range(OH):
         for ow in range(OW):
             cols[:, oh, ow] = padded[:, oh * stride:oh * stride + KH, ow * stride:ow * stride + KW, :]
+    if run_pad:
+        runs = np.zeros((B * OH * OW, KH, round_up(KW * c_pad, 16)), dtype=In.dtype)
+        runs[:, :, :KW * c_pad] = cols.reshape(B * OH * OW, KH, KW * c_pad)
+        return runs.reshape(B * OH * OW, -1)
     return cols.reshape(B * OH * OW, KH * KW * c_pad)
 
 
@@ -53,8 +58,12 @@ def device_weights(qb, case, fmt):
         Wp = np.zeros((OC, KH * KW, cp), dtype=np.int32)
         Wp[:, :, :C] = case.Wt.reshape(OC, KH * KW, C)
         flat = Wp.reshape(OC, -1)
-    else:
+    elif C % 16 == 0:
         flat = case.Wt.reshape(OC, -1)
+    else:                       # one zero-padded run per filter row
+        runs = np.zeros((OC, KH, round_up(KW * C, 16)), dtype=np.int32)
+        runs[:, :, :KW * C] = case.Wt.reshape(OC, KH, KW * C)
+        flat = runs.reshape(OC, -1)
     return qb.pack(qb.to_device_logical(flat, case.w_enc), case.w_bits, case.w_enc, fmt)
 
 
@@ -90,7 +99,8 @@ def test_im2col_matches_host_lowering(qb, fmt, shape):
         want = host_im2col(case.In, case.KH, case.KW, case.stride, case.pad, round_up(case.C, 32))
     else:
         got = unpack_int8(low.cpu().numpy(), npix, K, case.a_enc)
-        want = host_im2col(case.In, case.KH, case.KW, case.stride, case.pad, case.C)
+        want = host_im2col(case.In, case.KH, case.KW, case.stride, case.pad, case.C,
+                           run_pad=case.C % 16 != 0)
     assert np.array_equal(got, want)
 
 
@@ -230,8 +240,7 @@ def test_alexnet_chain_graph_replay(qb):
 ])
 def test_byte_lowering_with_contiguous_pixels_and_padding(qb, shape):
     """Pixel pitch == C (no per-pixel padding) with zero padding around the image: the
-    staged byte lowering (unaligned-word reads and the byte-by-byte path for words that
-    straddle two filter rows) against the host lowering and the direct convolution."""
+    run-per-filter-row byte lowering against the host lowering and the direct convolution."""
     case = synth.conv_case(970 + shape[3], *shape, w_enc=synth.SIGNED, a_enc=synth.UNSIGNED)
     x, pitch = device_map(qb, case, INT8, in_pitch=case.C)
     d = conv_desc(qb, case, INT8, INT8, pitch)
@@ -240,7 +249,7 @@ def test_byte_lowering_with_contiguous_pixels_and_padding(qb, shape):
     qb.check(qb.qnn_im2col(d, x, low))
     torch.cuda.synchronize()
     got = unpack_int8(low.cpu().numpy(), npix, qb.qnn_conv_lowered_k(d), case.a_enc)
-    want = host_im2col(case.In, case.KH, case.KW, case.stride, case.pad, case.C)
+    want = host_im2col(case.In, case.KH, case.KW, case.stride, case.pad, case.C, run_pad=True)
     assert np.array_equal(got, want)
     Wp = device_weights(qb, case, INT8)
     out = qb.qconv(d, Wp, x, torch.from_numpy(case.thr).cuda())

@@ -87,11 +87,12 @@ def test_conv_geometry(qb):
     d.fmt = 1
     assert qb.qnn_conv_lowered_k(d) == 2400
     assert qb.qnn_conv_lowered_bytes(d) == 729 * 2400
-    # conv1: 227x227x3, 11x11 stride 4 -> (96, 363, 3025), row pitch 368
+    # conv1: 227x227x3, 11x11 stride 4 -> (96, 363, 3025); each filter row (33 bytes) is a
+    # run padded to 48 bytes, so the lowered depth is 11 * 48
     d = qb.qnn_conv_desc(1, 227, 227, 3, 3, 96, 11, 11, 4, 0, 8, 8, 2, 1, 0, 1, 1, 0)
     assert qb.qnn_conv_out_h(d) == 55
-    assert qb.qnn_conv_lowered_k(d) == 363
-    assert qb.qnn_conv_lowered_bytes(d) == 3025 * 368
+    assert qb.qnn_conv_lowered_k(d) == 11 * 48
+    assert qb.qnn_conv_lowered_bytes(d) == 3025 * 528
     # channel count not a multiple of 32: every pixel is padded to whole words
     d = qb.qnn_conv_desc(1, 8, 8, 40, 0, 16, 3, 3, 1, 1, 1, 2, 2, 2, 0, 0, 1, 0)
     assert qb.qnn_conv_lowered_k(d) == 32 * 9 * 2

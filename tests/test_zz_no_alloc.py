@@ -43,7 +43,11 @@ def _setup(qb, case, fmt):
         m = np.zeros((B, H, Wd, pitch), dtype=np.uint8)
         m[..., :C] = case.In.astype(np.uint8)
         x = torch.from_numpy(m).cuda()
-        Wl = case.Wt
+        if C % 16 == 0:
+            Wl = case.Wt
+        else:                   # 8-bit maps with other channel counts: one zero-padded run per filter row
+            Wl = np.zeros((OC, KH, (KW * C + 15) // 16 * 16), dtype=np.int32)
+            Wl[:, :, :KW * C] = case.Wt.reshape(OC, KH, KW * C)
     Wp = qb.pack(qb.to_device_logical(Wl.reshape(OC, -1), case.w_enc), case.w_bits, case.w_enc, fmt)
     d = qb.qnn_conv_desc(B, H, Wd, C, pitch, OC, KH, KW, case.stride, case.pad, case.w_bits,
                          case.a_bits, case.out_bits, case.w_enc, case.a_enc, fmt, INT8, 0)
