@@ -1075,7 +1075,7 @@ struct TcPlan {
     bool share;
 };
 
-static bool tc_plan(const qnn_gemm_desc *d, int sms, TcPlan *pl) {
+static bool tc_plan(const qnn_gemm_desc *d, int sms, int num_kb, TcPlan *pl) {
     // channel tile: the widest that still gives every SM a tile
     const int tiles_p = ceil_div(d->N, TC_BP);
     int bn = 256;
@@ -1089,8 +1089,15 @@ static bool tc_plan(const qnn_gemm_desc *d, int sms, TcPlan *pl) {
     // sharing: a partial last round on at most half of an even number of SMs; the landing
     // zone is the weight ring (bn x 512 bytes of sums fit STAGES >= 4 stages of bn x 128 bytes)
     const char *no_share = getenv("QNN_TC_NO_SHARE");
-    pl->share = pl->rem > 0 && 2 * pl->rem <= pl->grid && (pl->grid % 2) == 0 && bn >= 128 &&
-                ceil_div(d->K, TC_BK) >= 2 && !(no_share && no_share[0] == '1');
+    const bool allowed = !(no_share && no_share[0] == '1');
+    pl->share = allowed && pl->rem > 0 && 2 * pl->rem <= pl->grid && (pl->grid % 2) == 0 && num_kb >= 2;
+    // Few tiles (at most half of the SMs): the kernel's time is the latency of one tile's serial
+    // depth loop, so every tile is shared by a CTA pair and each CTA walks half of the depth.
+    if (allowed && !pl->share && 2 * tiles <= sms && num_kb >= 4) {
+        pl->share = true;
+        pl->rem = (int)tiles;
+        pl->grid = 2 * (int)tiles;
+    }
     return true;
 }
 
@@ -1134,12 +1141,12 @@ static qnn_status tc_launch(const qnn_gemm_desc *d, const qnn_conv_desc *cv, con
         return launch_pair_out(mode, d->out_bits, ma, mw, p, s);
     }
     TcPlan pl;
-    if (!tc_plan(d, sms, &pl)) return QNN_ERR_UNSUPPORTED;
+    if (!tc_plan(d, sms, p.num_kb, &pl)) return QNN_ERR_UNSUPPORTED;
     const int bn = pl.bn;
     p.tiles_p = pl.tiles_p; p.tiles_c = pl.tiles_c;
     const int tiles = pl.tiles_p * pl.tiles_c;
     p.units = p.full_units = tiles;
-    if (pl.share) {
+    if (pl.share) {                       // the last pl.rem tiles (possibly all) are shared by CTA pairs
         p.share = 1;
         p.full_units = tiles - pl.rem;
         p.units = p.full_units + 2 * pl.rem;
@@ -1178,7 +1185,7 @@ qnn_status gemm_tc_conv_launch(const qnn_conv_desc *cv, const qnn_gemm_desc *g, 
     // count is not a multiple of 128 that loop has more (partly empty) k-blocks here than over the
     // dense lowered matrix, so small problems keep the explicit lowering.
     TcPlan pl;
-    if (!tc_plan(g, sm_count(), &pl)) return QNN_ERR_UNSUPPORTED;
+    if (!tc_plan(g, sm_count(), ceil_div(g->K, TC_BK), &pl)) return QNN_ERR_UNSUPPORTED;
     const long long tiles = (long long)pl.tiles_p * pl.tiles_c;
     const char *force = getenv("QNN_CONV_IMPLICIT");          // "1": skip this heuristic (tests)
     if (!(force && force[0] == '1') && tiles <= sm_count() &&
