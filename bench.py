@@ -316,10 +316,15 @@ def run_b200(args):
     qdist.finalize()
 
 
+QUICK = False      # --quick: few iterations and no graph replay (profiler captures)
+
+
 def _time_calls(torch, fn, iters, warmup=3, graph=False):
     """Mean device milliseconds of fn(i), CUDA events on the current stream.  With graph=True
     the `iters` calls are recorded into one CUDA graph and the graph is replayed, which takes
     the host's per-call cost (a few microseconds of Python and ctypes) out of the number."""
+    if QUICK:
+        iters, warmup, graph = min(iters, 2), 1, False
     for i in range(warmup):
         fn(i)
     torch.cuda.synchronize()
@@ -361,10 +366,11 @@ def run_extras(args):
     PL, I8 = qb.QNN_FMT_BITPLANES, qb.QNN_FMT_INT8
     res = {"workload": "extras", "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"]}
 
+    only = args.extras_only
     # ---- config 5: M = K = 8192, N in {1, 4, 16}; W2A2 and W4A4
     M = K = 8192
     skinny = []
-    for bits in (2, 4):
+    for bits in (2, 4) if only in (None, "skinny") else ():
         c = synth.gemm_case(5000 + bits, M, 16, K, bits, bits)
         Wd = qb.to_device_logical(c.W, c.w_enc)
         thr = torch.from_numpy(c.thr).cuda()
@@ -389,7 +395,7 @@ def run_extras(args):
 
     # ---- config 3: conv2-shaped W1A2 layer via lowering, B = 1 and 64
     conv = []
-    for B in (1, 64):
+    for B in (1, 64) if only in (None, "conv2") else ():
         c = synth.conv2_alexnet_case(B)
         for fmt, name in ((I8, "int8"), (PL, "bitplanes")):
             if fmt == PL:
@@ -414,7 +420,7 @@ def run_extras(args):
 
     # ---- config 4: AlexNet-shaped chain, B = 1 and 256
     net_res = []
-    for B in (1, 256):
+    for B in ((1, 256) if not QUICK else (32,)) if only in (None, "alexnet") else ():
         net = synth.alexnet_case(B)
         for mode in ("auto", "tensor", "bitserial") if B == 1 else ("auto",):
             plan = AlexNetPlan(net, B, mode)
@@ -434,9 +440,12 @@ def run_extras(args):
                     f = lambda i: qb.check(qb.qnn_qgemm(d, Wp, x_in, thr, out, None, 0))
                 per_layer[name] = round(1e3 * _time_calls(torch, f, 20, graph=True), 2)
                 prev = out
-            graph, _ = plan.capture(img)
-            ms_graph = _time_calls(torch, lambda i: graph.replay(), 30 if B == 1 else 10)
-            del graph
+            if QUICK:
+                ms_graph = ms
+            else:
+                graph, _ = plan.capture(img)
+                ms_graph = _time_calls(torch, lambda i: graph.replay(), 30 if B == 1 else 10)
+                del graph
             net_res.append({"B": B, "mode": mode, "ms": ms, "images_per_s": B / ms * 1e3,
                             "ms_graph": ms_graph, "images_per_s_graph": B / ms_graph * 1e3,
                             "launches": plan.launches_per_forward(), "per_layer_us": per_layer})
@@ -462,6 +471,10 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--overlap", type=int, default=1,
                     help="1: activation packer on a second stream, overlapping the previous GEMM (default); 0: one stream")
+    ap.add_argument("--extras-only", default=None, choices=["skinny", "conv2", "alexnet"],
+                    help="extras: run one group only")
+    ap.add_argument("--quick", action="store_true",
+                    help="extras: a couple of plain calls per case (for profiler captures; AlexNet at batch 32)")
     ap.add_argument("--workload", default="sweep", choices=["sweep", "extras"],
                     help="sweep: the headline line; extras: the other paper-shaped workloads (one GPU)")
     ap.add_argument("--pairs", default=None,
@@ -470,6 +483,8 @@ def main():
     if args.pairs:
         PAIRS[:] = [tuple(int(v) for v in p.split("x")) for p in args.pairs.split(",")]
     if args.workload == "extras":
+        global QUICK
+        QUICK = args.quick
         run_extras(args)
         return
     if args.impl == "reference":
