@@ -289,6 +289,23 @@ def run_b200(args):
                "sample": f"first {rows} weight rows x all {DIM} columns, K={DIM}, (w,a) in {pairs}: "
                          f"{m:.3g} MAC in {s:.1f} s"}
 
+    # ---- second half of the metric: AlexNet-shaped W1A2 chain, images/s (N = 1 only)
+    alexnet = None
+    if world == 1 and not args.no_alexnet:
+        from paper_1709_04060_b200.alexnet import AlexNetPlan
+        alexnet = {}
+        for B in (256, 1):
+            net = synth.alexnet_case(B)
+            plan = AlexNetPlan(net, B, "auto")
+            img = torch.from_numpy(net.image.astype(np.uint8)).cuda()
+            graph, _ = plan.capture(img)
+            ms_b = _time_calls(torch, lambda i: graph.replay(), 20 if B > 1 else 50)
+            alexnet[f"batch{B}"] = {"images_per_s": B / ms_b * 1e3, "ms": ms_b,
+                                    "kernels_per_forward": plan.launches_per_forward()}
+            del graph, plan
+        alexnet["note"] = ("random-init AlexNet-shaped W1A2 chain (conv1/fc8 8-bit), uint8 images resident "
+                           "in HBM, one CUDA-graph replay per forward pass")
+
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
@@ -310,6 +327,7 @@ def run_b200(args):
                      "peak_source": f"2 x {peaks['source']} bf16 sustained cuBLAS TFLOP/s (nominal int8:bf16 ratio)",
                      "avg_launch_ms": gemm_avg_ms, "algorithmic_ops_per_launch": 2.0 * DIM ** 3},
         "per_pair_tmacs": per_pair,
+        "alexnet_w1a2": alexnet,
         "cpu_baseline": cpu,
     }
     print(json.dumps(out))
@@ -469,6 +487,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-alexnet", action="store_true", help="skip the AlexNet-shaped chain measurement")
     ap.add_argument("--overlap", type=int, default=1,
                     help="1: activation packer on a second stream, overlapping the previous GEMM (default); 0: one stream")
     ap.add_argument("--extras-only", default=None, choices=["skinny", "conv2", "alexnet"],

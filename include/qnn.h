@@ -213,6 +213,32 @@ typedef struct {
 /* out has the same format with H, W replaced by (H-k)/stride+1, (W-k)/stride+1. */
 qnn_status qnn_maxpool(const qnn_pool_desc *d, const void *in, void *out, void *stream);
 
+/* ---- streamlining (Section 2.1), host only -------------------------------- */
+
+/* Float parameters around one output channel of a quantized matrix layer. */
+typedef struct {
+    double a_prev, b_prev;     /* previous layer's activation value = a_prev * code + b_prev
+                                  (quantizer as thresholding + affine map, Section 2.1.1) */
+    double alpha;              /* alpha-scaling of this channel's weight row (Section 2) */
+    double gamma, beta;        /* batch normalisation: gamma * (z - mu) / sigma + beta     */
+    double mu, sigma;
+    long long row_sum;         /* sum of the channel's integer weights: the W.b term of
+                                  W.(a x + b) = a (W.x) + W.b (Section 2.1.2)              */
+} qnn_channel_params;
+
+/* Absorbs the float operations between the integer accumulator and the activation
+ * quantizer into integer thresholds (Sections 2.1.2 and 2.1.3).  qthr: the quantizer's
+ * n_thr float thresholds, ascending (e.g. {0, 0.807, 1.345} for the 2-bit HWGQ quantizer);
+ * [acc_lo, acc_hi]: range of the accumulator (|.| < 2^31).  thr_out [channels][n_thr]:
+ * threshold i is the smallest integer accumulator whose float forward pass reaches code
+ * i + 1, INT32_MIN if every accumulator does, INT32_MAX if none does; a tie (accumulator
+ * maps exactly onto a float threshold) counts as passed.  negate_out [channels]: 1 where
+ * the collapsed slope is negative -- that channel's thresholds are for the NEGATED
+ * accumulator, i.e. the caller negates the channel's weight row.  All pointers are host
+ * pointers; nothing is launched.  Errors: INVALID_ARG. */
+qnn_status qnn_streamline(const qnn_channel_params *ch, int channels, const double *qthr, int n_thr,
+                          long long acc_lo, long long acc_hi, int32_t *thr_out, uint8_t *negate_out);
+
 /* ---- utilities ------------------------------------------------------------ */
 
 /* Checks on the device that every row of thr [M][n_thr] is sorted

@@ -36,7 +36,7 @@ EXPORTS = (
     "qnn_gemm_out_bytes", "qnn_qgemm", "qnn_conv_out_h", "qnn_conv_out_w",
     "qnn_conv_lowered_k", "qnn_conv_lowered_bytes", "qnn_conv_workspace_bytes",
     "qnn_conv_out_bytes", "qnn_im2col", "qnn_qconv", "qnn_qconv_static", "qnn_maxpool",
-    "qnn_validate_thresholds", "qnn_device_status", "qnn_launch_count",
+    "qnn_streamline", "qnn_validate_thresholds", "qnn_device_status", "qnn_launch_count",
     "qnn_status_string", "qnn_version",
 )
 
@@ -55,6 +55,11 @@ class qnn_conv_desc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in (
         "B", "H", "W", "C", "in_pitch", "OC", "KH", "KW", "stride", "pad",
         "w_bits", "a_bits", "out_bits", "w_enc", "a_enc", "fmt", "out_fmt", "path")]
+
+
+class qnn_channel_params(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_double) for n in ("a_prev", "b_prev", "alpha", "gamma", "beta", "mu", "sigma")] + \
+               [("row_sum", ctypes.c_longlong)]
 
 
 class qnn_pool_desc(ctypes.Structure):
@@ -91,6 +96,9 @@ _lib.qnn_qconv_static.restype = _ci
 _lib.qnn_qconv_static.argtypes = [_P(qnn_conv_desc), _vp, _vp, _vp, _vp, _vp]
 _lib.qnn_maxpool.restype = _ci
 _lib.qnn_maxpool.argtypes = [_P(qnn_pool_desc), _vp, _vp, _vp]
+_lib.qnn_streamline.restype = _ci
+_lib.qnn_streamline.argtypes = [_P(qnn_channel_params), _ci, _P(ctypes.c_double), _ci, ctypes.c_longlong,
+                                ctypes.c_longlong, _P(ctypes.c_int32), _P(ctypes.c_uint8)]
 _lib.qnn_validate_thresholds.restype = _ci
 _lib.qnn_validate_thresholds.argtypes = [_vp, _ci, _ci, _P(_ci), _vp]
 _lib.qnn_device_status.restype = _ci
@@ -214,6 +222,21 @@ def qnn_qconv_static(d, Wpacked, inp, thr, out, stream=None) -> int:
 
 def qnn_maxpool(d, inp, out, stream=None) -> int:
     return _lib.qnn_maxpool(ctypes.byref(d), _ptr(inp), _ptr(out), _stream(stream))
+
+
+def qnn_streamline(channels, qthr, acc_lo: int, acc_hi: int):
+    """Host-only.  channels: sequence of qnn_channel_params (or 8-tuples in field order);
+    qthr: the quantizer's float thresholds.  Returns (status, thresholds [channels][n_thr] as
+    nested lists of ints, negate flags)."""
+    arr = (qnn_channel_params * len(channels))(*[c if isinstance(c, qnn_channel_params) else qnn_channel_params(*c)
+                                                  for c in channels])
+    n = len(qthr)
+    q = (ctypes.c_double * n)(*[float(t) for t in qthr])
+    out = (ctypes.c_int32 * (len(channels) * n))()
+    neg = (ctypes.c_uint8 * len(channels))()
+    st = _lib.qnn_streamline(arr, len(channels), q, n, int(acc_lo), int(acc_hi), out, neg)
+    thr = [[out[c * n + i] for i in range(n)] for c in range(len(channels))]
+    return st, thr, [int(v) for v in neg]
 
 
 def qnn_validate_thresholds(thr, M: int, n_thr: int, stream=None):

@@ -281,3 +281,31 @@ def test_skinny_byte_kernel_encodings(qb, w_enc, a_enc, w, a):
         run_case(qb, case, INT8, INT8, check_pack=True)
         run_case(qb, case, INT8, BITPLANES)
         run_case(qb, case, INT8, INT8, raw=True)
+
+
+def test_streamlined_layer_end_to_end(qb):
+    """Section 2.1 end to end: float alpha / batch-norm / quantizer parameters of a W1A2 layer
+    are absorbed into integer thresholds by the library's host tool (rows with a negative
+    collapsed slope are negated), the fused GEMM+threshold kernel runs on integers only, and its
+    codes equal the float forward pass of the un-streamlined layer evaluated by the oracle."""
+    from oracle import streamline as ref
+    case = synth.gemm_case(7000, 64, 256, 576, 1, 2)
+    rng = np.random.default_rng(7000)
+    chans = [ref.random_params(rng, int(case.W[m].sum()), 45.0) for m in range(64)]
+    st, thr, neg = qb.qnn_streamline(
+        [(c.a_prev, c.b_prev, c.alpha, c.gamma, c.beta, c.mu, c.sigma, c.row_sum) for c in chans],
+        ref.HWGQ_THRESHOLDS, -1728, 1728)
+    assert st == 0 and any(neg)
+    W_dev = case.W.copy()
+    W_dev[np.array(neg, dtype=bool)] *= -1                       # bipolar rows: a sign flip
+    acc = orc.gemm(case.W, case.At)                              # accumulators of the original layer
+    want = np.array([[ref.float_forward(int(acc[m, n]), chans[m], ref.HWGQ_THRESHOLDS)
+                      for m in range(64)] for n in range(256)])
+    for fmt in (INT8, BITPLANES):
+        Wp = qb.pack(qb.to_device_logical(W_dev, case.w_enc), 1, case.w_enc, fmt)
+        Ap = qb.pack(qb.to_device_logical(case.At, case.a_enc), 2, case.a_enc, fmt)
+        d = qb.gemm_desc(64, 256, 576, 1, 2, 2, case.w_enc, case.a_enc, fmt, INT8)
+        out = qb.qgemm(d, Wp, Ap, torch.tensor(thr, dtype=torch.int32).cuda())
+        torch.cuda.synchronize()
+        got = decode_out(out.cpu().numpy(), INT8, 2, 256, 64, False)
+        assert np.array_equal(got, want)
