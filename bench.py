@@ -474,6 +474,48 @@ def run_extras(args):
     print(json.dumps(res))
 
 
+def run_shapes(args):
+    """Size sweep of Section 4.1.2 of the paper: every (rows, depth, cols) in {2^6 .. 2^12}^3 for
+    W1A1 (bipolar x bipolar) GEMM+threshold, on 8-bit containers (tensor cores, or byte dot
+    products below 9 columns) and on bit planes (bit-serial kernels), each timed by replaying a
+    CUDA graph of repeated calls.  Prints one JSON line with the per-shape times and the faster
+    operand format."""
+    import torch
+    import __graft_entry__ as ge
+    ge.build()
+    from paper_1709_04060_b200 import binding as qb
+    torch.cuda.set_device(0)
+    PL, I8, BIP = qb.QNN_FMT_BITPLANES, qb.QNN_FMT_INT8, qb.QNN_ENC_BIPOLAR
+    dims = [2 ** e for e in range(6, 13)]
+    if QUICK:
+        dims = [64, 1024, 4096]
+    g = torch.Generator(device="cuda").manual_seed(170904060)
+    big = (2 * torch.randint(0, 2, (4096, 4096), dtype=torch.int8, device="cuda", generator=g) - 1).contiguous()
+    thr_all = torch.randint(-32, 33, (4096, 1), dtype=torch.int32, device="cuda", generator=g)
+    rows = []
+    for M in dims:
+        for K in dims:
+            Wl = big[:M, :K].contiguous()
+            Wp = {f: qb.pack(Wl, 1, BIP, f) for f in (I8, PL)}
+            thr = thr_all[:M].contiguous()
+            for N in dims:
+                Al = big[4096 - N:, 4096 - K:].contiguous()
+                res = {"M": M, "K": K, "N": N}
+                for f, name in ((I8, "int8"), (PL, "bitplanes")):
+                    Ap = qb.pack(Al, 1, BIP, f)
+                    d = qb.gemm_desc(M, N, K, 1, 1, 1, BIP, BIP, f, I8)
+                    out = torch.empty(max(qb.qnn_gemm_out_bytes(d, True), 16), dtype=torch.uint8, device="cuda")
+                    reps = 10 if M * N * K < 2 ** 30 else 3
+                    ms = _time_calls(torch, lambda i: qb.check(qb.qnn_qgemm(d, Wp[f], Ap, thr, out)), reps, graph=True)
+                    res[name + "_us"] = round(1e3 * ms, 2)
+                res["gmacs_best"] = round(M * N * K / (min(res["int8_us"], res["bitplanes_us"]) * 1e-6) / 1e9, 1)
+                res["faster"] = "int8" if res["int8_us"] <= res["bitplanes_us"] else "bitplanes"
+                rows.append(res)
+    n_bit = sum(r["faster"] == "bitplanes" for r in rows)
+    print(json.dumps({"workload": "shapes", "precision": "W1A1 bipolar, 1 threshold per row", "shapes": len(rows),
+                      "bitplanes_faster": n_bit, "rows": rows}))
+
+
 # dram__bytes_read.sum + dram__bytes_write.sum of one 4096^3 W1A2 launch of the tensor-core
 # kernel, from the ncu capture summarised in profiles/qgemm_tc_4096_w1a2_w4a4.md (the output
 # codes were still in L2 when the capture ended, so the write counter is small).
@@ -494,17 +536,18 @@ def main():
                     help="extras: run one group only")
     ap.add_argument("--quick", action="store_true",
                     help="extras: a couple of plain calls per case (for profiler captures; AlexNet at batch 32)")
-    ap.add_argument("--workload", default="sweep", choices=["sweep", "extras"],
-                    help="sweep: the headline line; extras: the other paper-shaped workloads (one GPU)")
+    ap.add_argument("--workload", default="sweep", choices=["sweep", "extras", "shapes"],
+                    help="sweep: the headline line; extras: the other paper-shaped workloads (one GPU); "
+                         "shapes: the 2^6..2^12 size sweep of both operand formats")
     ap.add_argument("--pairs", default=None,
                     help="restrict the sweep, e.g. '1x2,4x4' (profiling only; the default is all 16)")
     args = ap.parse_args()
     if args.pairs:
         PAIRS[:] = [tuple(int(v) for v in p.split("x")) for p in args.pairs.split(",")]
-    if args.workload == "extras":
+    if args.workload in ("extras", "shapes"):
         global QUICK
         QUICK = args.quick
-        run_extras(args)
+        (run_extras if args.workload == "extras" else run_shapes)(args)
         return
     if args.impl == "reference":
         if args.steps is None:

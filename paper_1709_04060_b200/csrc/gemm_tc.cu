@@ -1076,11 +1076,33 @@ struct TcPlan {
 };
 
 static bool tc_plan(const qnn_gemm_desc *d, int sms, int num_kb, TcPlan *pl) {
-    // channel tile: the widest that still gives every SM a tile
+    const char *no_share = getenv("QNN_TC_NO_SHARE");
+    const bool allowed = !(no_share && no_share[0] == '1');
+    // Channel tile.  An MMA costs about the same for every N (measured: the 128 x 32-byte
+    // activation operand bounds it), so a tile's main loop costs num_kb k-blocks whatever its
+    // width; a narrower tile only shortens the epilogue of the last tile and adds rounds.  Pick the
+    // width with the smallest estimated time: rounds x max(main loop, epilogue) + one exposed
+    // epilogue, in cycles (about 640 per k-block, 2000 per 32-column chunk and epilogue warp).
     const int tiles_p = ceil_div(d->N, TC_BP);
-    int bn = 256;
-    while (bn > 32 && (bn / 2 >= round_up(d->M, 32) || (long long)tiles_p * ceil_div(d->M, bn) < sms)) bn >>= 1;
-    if (bn == 64) bn = 32;
+    const int cand[3] = {256, 128, 32};
+    double best_cost = 0.0;
+    int bn = 0;
+    for (int ci = 0; ci < 3; ++ci) {
+        const int b = cand[ci];
+        if (b > 32 && b / 2 >= round_up(d->M, 32)) continue;        // wider than the channels need
+        const long long t = (long long)tiles_p * ceil_div(d->M, b);
+        const double main_loop = 640.0 * num_kb, epi = 2000.0 * (b >= 64 ? b / 64 : 1);
+        double cost;
+        if (allowed && 2 * t <= sms && num_kb >= 4) {
+            cost = 0.5 * main_loop + 1000.0 + epi;                   // every tile shared by a CTA pair
+        } else {
+            const long long full = t / sms, rem = t % sms;
+            double rounds = (double)full;
+            if (rem > 0) rounds += (allowed && full > 0 && 2 * rem <= sms && (sms % 2) == 0 && num_kb >= 2) ? 0.55 : 1.0;
+            cost = rounds * (main_loop > epi ? main_loop : epi) + epi;
+        }
+        if (bn == 0 || cost < best_cost) { bn = b; best_cost = cost; }
+    }
     pl->bn = bn; pl->tiles_p = tiles_p; pl->tiles_c = ceil_div(d->M, bn);
     const long long tiles = (long long)pl->tiles_p * pl->tiles_c;
     if (tiles > 0x3fffffff) return false;
@@ -1088,8 +1110,6 @@ static bool tc_plan(const qnn_gemm_desc *d, int sms, int num_kb, TcPlan *pl) {
     pl->rem = (int)(tiles % pl->grid);
     // sharing: a partial last round on at most half of an even number of SMs; the landing
     // zone is the weight ring (bn x 512 bytes of sums fit STAGES >= 4 stages of bn x 128 bytes)
-    const char *no_share = getenv("QNN_TC_NO_SHARE");
-    const bool allowed = !(no_share && no_share[0] == '1');
     pl->share = allowed && pl->rem > 0 && 2 * pl->rem <= pl->grid && (pl->grid % 2) == 0 && num_kb >= 2;
     // Few tiles (at most half of the SMs): the kernel's time is the latency of one tile's serial
     // depth loop, so every tile is shared by a CTA pair and each CTA walks half of the depth.
