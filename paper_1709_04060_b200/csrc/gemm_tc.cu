@@ -1193,14 +1193,13 @@ qnn_status gemm_tc_launch(const qnn_gemm_desc *d, const void *W, const void *A, 
 }
 
 // Convolution without a lowered matrix: the GEMM's loader reads the 8-bit channels-last map
-// through an im2col tensor map.  UNSUPPORTED when the shape needs the explicit lowering
-// (channel count or pixel pitch not a multiple of 16, stride other than 1).
+// through an im2col tensor map (base pixels step by the stride).  UNSUPPORTED when the shape
+// needs the explicit lowering (channel count or pixel pitch not a multiple of 16).
 qnn_status gemm_tc_conv_launch(const qnn_conv_desc *cv, const qnn_gemm_desc *g, const void *W, const void *in,
                                const int32_t *thr, void *out, cudaStream_t s) {
     const int pitch = cv->in_pitch ? cv->in_pitch : round_up(cv->C, 16);
-    if (cv->fmt != QNN_FMT_INT8 || (cv->C % 16) != 0 || (pitch % 16) != 0 || cv->stride != 1)
-        return QNN_ERR_UNSUPPORTED;
-    if (cv->KH > 255 || cv->KW > 255) return QNN_ERR_UNSUPPORTED;
+    if (cv->fmt != QNN_FMT_INT8 || (cv->C % 16) != 0 || (pitch % 16) != 0) return QNN_ERR_UNSUPPORTED;
+    if (cv->KH > 255 || cv->KW > 255 || cv->stride > 8) return QNN_ERR_UNSUPPORTED;
     // A single round of tiles is bound by the latency of its serial depth loop.  When the channel
     // count is not a multiple of 128 that loop has more (partly empty) k-blocks here than over the
     // dense lowered matrix, so small problems keep the explicit lowering.

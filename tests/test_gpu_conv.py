@@ -298,6 +298,9 @@ def test_config4_alexnet_batch256_sampled_images(qb):
     (5, 6, 7, 48, 40, 3, 2, 1, 0, 2, 2),          # no padding, ragged everything
     (1, 5, 5, 272, 33, 5, 5, 1, 4, 3, 3),         # padding larger than half the filter, 128+128+16 bytes
     (200, 4, 4, 16, 70, 2, 2, 1, 1, 4, 4),        # many small images: tiles span several images
+    (3, 12, 12, 32, 64, 3, 3, 2, 0, 1, 2),        # stride 2, no padding
+    (2, 23, 17, 64, 48, 5, 3, 3, 2, 2, 2),        # stride 3 with padding, rectangular filter and image
+    (4, 9, 9, 128, 130, 3, 3, 2, 1, 1, 2),        # stride 2, padding 1, a full 128-byte chunk
 ])
 def test_implicit_convolution_shapes(qb, monkeypatch, shape):
     """Convolution with the lowering done by the tensor-core kernel's loader, against the direct
