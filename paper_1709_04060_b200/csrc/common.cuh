@@ -28,6 +28,22 @@ inline qnn_status launch_status() {
     return cudaGetLastError() == cudaSuccess ? QNN_OK : QNN_ERR_CUDA;
 }
 
+// Programmatic dependent launch.  The tensor-core GEMM, when its grid fills the GPU, is launched
+// so that its CTAs may be placed while the previous kernel of the stream drains (they wait in
+// griddepcontrol.wait before touching global memory).  The other kernels only do their part as
+// predecessors: pdl_trigger() tells the scheduler that a dependent may start placing CTAs (no
+// effect unless the next kernel asked for it), pdl_wait() is a no-op for a normally launched
+// kernel.  They are not launched that way themselves: early placement next to a draining kernel
+// packs the CTAs of a small grid onto few SMs, which halved the bit-serial kernel's speed.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_enter() {
+    pdl_trigger();
+    pdl_wait();
+}
+#endif
+
 // Number of SMs of the current device (cached per device).
 int sm_count();
 

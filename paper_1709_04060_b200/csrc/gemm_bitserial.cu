@@ -43,6 +43,7 @@ qgemm_bitserial_kernel(const BsParams p) {
     __shared__ uint32_t As[AB][BS_BN][BS_PITCH];
     __shared__ int corr_s[64];
 
+    pdl_wait();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int m0 = blockIdx.y * BS_BM, n0 = blockIdx.x * BS_BN;
     const int lc = tid & 15, lr = tid >> 4;      // staging: word column, first row
@@ -105,6 +106,8 @@ qgemm_bitserial_kernel(const BsParams p) {
         }
         __syncthreads();
     }
+
+    pdl_trigger();          // main loop done: the next kernel may start placing its CTAs
 
     // correction sums: reduce the 16 staging threads that share a row
     if (MODE == BS_W_BIPOLAR || MODE == BS_A_BIPOLAR) {

@@ -641,6 +641,10 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
     if (p.share) cluster_sync_all();       // the peer's barriers are initialised before anyone signals them
     else __syncthreads();
     tc_fence_after();
+    // set-up done: a kernel queued behind this one may start placing CTAs as SMs fall idle, and
+    // this one waits here for the kernel before it (no global memory has been touched yet)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint32_t tmem_base = sm.tmem_base;
     if (threadIdx.x == 0) QNN_TRACE(4, 1);
 
@@ -1000,19 +1004,28 @@ static qnn_status launch_cfg(const CUtensorMap &ma, const CUtensorMap &mw, const
         attr_done = true;
     }
     const int grid = p.units < sm_count() ? p.units : sm_count();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(TC_THREADS);
+    cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute attr[2];
+    int na = 0;
+    // Programmatic dependent launch: when the previous operation on the stream is a kernel that
+    // has released its dependents, this kernel's CTAs may start on SMs as they fall idle and do
+    // their set-up there; they touch no global memory before griddepcontrol.wait, which returns
+    // once the previous kernel has completed.
+    if (grid >= sm_count()) {        // small grids: early placement only crowds the idle SMs
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
     if (p.share) {
         // clusters of two CTAs: consecutive block indices share a tile of the last round
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(grid); cfg.blockDim = dim3(TC_THREADS);
-        cfg.dynamicSmemBytes = smem; cfg.stream = s;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr; cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, kern, ma, mw, p) != cudaSuccess) return QNN_ERR_CUDA;
-    } else {
-        kern<<<grid, TC_THREADS, smem, s>>>(ma, mw, p);
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = 2; attr[na].val.clusterDim.y = 1; attr[na].val.clusterDim.z = 1;
+        ++na;
     }
+    cfg.attrs = attr; cfg.numAttrs = na;
+    if (cudaLaunchKernelEx(&cfg, kern, ma, mw, p) != cudaSuccess) return QNN_ERR_CUDA;
     count_launch();
     return launch_status();
 }

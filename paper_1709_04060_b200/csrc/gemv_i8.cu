@@ -37,6 +37,7 @@ template <bool W_SIGNED, bool A_SIGNED>
 __global__ void __launch_bounds__(G8_THREADS)
 gemv_i8_kernel(const G8Params p) {
     extern __shared__ __align__(16) uint8_t g8_smem[];     // [G8_COLS][ld] activation bytes
+    pdl_wait();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int n0 = blockIdx.y * G8_COLS;
     const int ncols = min(G8_COLS, p.N - n0);
@@ -100,9 +101,11 @@ gemv_i8_kernel(const G8Params p) {
             }
         }
     }
+    pdl_trigger();
 }
 
 __global__ void gemv_i8_clear_kernel(uint32_t *out, long long words) {
+    pdl_enter();
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < words;
          i += (long long)gridDim.x * blockDim.x)
         out[i] = 0u;

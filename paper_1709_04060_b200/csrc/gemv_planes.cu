@@ -35,6 +35,7 @@ __global__ void __launch_bounds__(GV_THREADS)
 gemv_planes_kernel(const GvParams p) {
     extern __shared__ uint32_t gv_smem[];          // [AB][GV_COLS][kw_pad] activation words
     __shared__ int corr_s[GV_COLS];
+    pdl_wait();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int n0 = blockIdx.y * GV_COLS;
     const int ncols = min(GV_COLS, p.N - n0);
@@ -165,11 +166,13 @@ gemv_planes_kernel(const GvParams p) {
             }
         }
     }
+    pdl_trigger();
 }
 
 // Clears the output before the kernel sets bits (bit-plane output) or leaves pad
 // bytes untouched (8-bit output: pad bytes of a row are zeroed here).
 __global__ void gemv_clear_kernel(uint32_t *out, long long words) {
+    pdl_enter();
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < words;
          i += (long long)gridDim.x * blockDim.x)
         out[i] = 0u;

@@ -45,6 +45,7 @@ template <> __device__ __forceinline__ uint4 zero_unit<uint4>() { return make_ui
 
 template <typename T>
 __global__ void __launch_bounds__(256) lower_units_kernel(const LowerParams p) {
+    pdl_enter();
     const int lane = threadIdx.x & 31;
     const long long warp0 = (blockIdx.x * (long long)blockDim.x + threadIdx.x) >> 5;
     const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
@@ -87,6 +88,7 @@ constexpr int LR_PIX = 64;
 __global__ void __launch_bounds__(256) lower_runs_kernel(const LowerParams p, int chunks, int span, int run,
                                                          int runp) {
     extern __shared__ __align__(16) uint8_t lr_smem[];   // [KH][seg_pitch] + slack
+    pdl_enter();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint8_t *in = reinterpret_cast<const uint8_t *>(p.in);
     const uint32_t *sm_words = reinterpret_cast<const uint32_t *>(lr_smem);

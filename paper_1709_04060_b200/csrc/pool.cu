@@ -18,6 +18,7 @@ struct PoolParams {
 
 // 16 channels (one uint4) per thread; the padded channel count is a multiple of 16.
 __global__ void __launch_bounds__(256) maxpool_u8_kernel(const PoolParams p) {
+    pdl_enter();
     const int cu = p.cu >> 2;                                     // 16-byte units per pixel
     const long long total = (long long)p.B * p.OH * p.OW * cu;
     const uint4 *in = reinterpret_cast<const uint4 *>(p.in);
@@ -43,6 +44,7 @@ __global__ void __launch_bounds__(256) maxpool_u8_kernel(const PoolParams p) {
 
 template <int BITS>
 __global__ void __launch_bounds__(256) maxpool_planes_kernel(const PoolParams p) {
+    pdl_enter();
     const long long total = (long long)p.B * p.OH * p.OW * p.cu;
     const uint32_t *in = reinterpret_cast<const uint32_t *>(p.in);
     uint32_t *out = reinterpret_cast<uint32_t *>(p.out);
