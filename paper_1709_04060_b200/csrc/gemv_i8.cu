@@ -43,11 +43,9 @@ gemv_i8_kernel(const G8Params p) {
     const int ncols = min(G8_COLS, p.N - n0);
     const int steps = p.ld >> 4;                           // 16-byte steps per row
 
-    for (int idx = threadIdx.x; idx < G8_COLS * steps; idx += G8_THREADS) {
+    for (int idx = threadIdx.x; idx < ncols * steps; idx += G8_THREADS) {      // only the columns in use
         const int c = idx / steps, q = idx - c * steps;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (c < ncols) v = reinterpret_cast<const uint4 *>(p.A + (size_t)(n0 + c) * p.ld)[q];
-        reinterpret_cast<uint4 *>(g8_smem)[idx] = v;
+        reinterpret_cast<uint4 *>(g8_smem)[idx] = reinterpret_cast<const uint4 *>(p.A + (size_t)(n0 + c) * p.ld)[q];
     }
     __syncthreads();
 
@@ -58,7 +56,7 @@ gemv_i8_kernel(const G8Params p) {
 #pragma unroll
         for (int c = 0; c < G8_COLS; ++c) acc[c] = 0;
         const uint4 *wrow = reinterpret_cast<const uint4 *>(p.W + (size_t)m * p.ld);
-#pragma unroll 4
+#pragma unroll 8
         for (int q = lane; q < steps; q += 32) {
             const uint4 w = __ldcs(wrow + q);
 #pragma unroll
@@ -138,7 +136,7 @@ qnn_status gemv_i8_launch(const qnn_gemm_desc *d, const void *W, const void *A,
             ++launches;
         }
     }
-    const size_t smem = (size_t)G8_COLS * p.ld;
+    const size_t smem = (size_t)(d->N < G8_COLS ? d->N : G8_COLS) * p.ld;    // only the columns in use
     const int row_blocks = ceil_div(d->M, G8_THREADS / 32);
     const int max_blocks = sm_count() * 8;
     dim3 grid(row_blocks < max_blocks ? row_blocks : max_blocks, ceil_div(d->N, G8_COLS));

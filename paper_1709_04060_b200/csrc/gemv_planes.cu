@@ -30,8 +30,10 @@ struct GvParams {
 
 enum { GV_REGULAR = 0, GV_W_BIPOLAR = 1, GV_A_BIPOLAR = 2, GV_BOTH_BIPOLAR = 3 };
 
+// At most 36 registers, so that 7 CTAs share an SM: the 1024 CTAs of an 8192-row layer are then
+// resident in a single wave (with more registers it took 1.4 waves, i.e. twice the latency chain).
 template <int WB, int AB, int MODE, bool VEC>
-__global__ void __launch_bounds__(GV_THREADS)
+__global__ void __launch_bounds__(GV_THREADS, 7)
 gemv_planes_kernel(const GvParams p) {
     extern __shared__ uint32_t gv_smem[];          // [AB][GV_COLS][kw_pad] activation words
     __shared__ int corr_s[GV_COLS];
@@ -44,11 +46,11 @@ gemv_planes_kernel(const GvParams p) {
     if (threadIdx.x < GV_COLS) corr_s[threadIdx.x] = 0;
     __syncthreads();
     for (int j = 0; j < AB; ++j)
-        for (int c = 0; c < GV_COLS; ++c) {
+        for (int c = 0; c < ncols; ++c) {                 // only the columns in use
             int part = 0;
             for (int d = threadIdx.x; d < p.kw_pad; d += GV_THREADS) {
                 uint32_t v = 0;
-                if (c < ncols && d < p.kw) v = p.A[((size_t)j * p.N + n0 + c) * p.kw + d];
+                if (d < p.kw) v = p.A[((size_t)j * p.N + n0 + c) * p.kw + d];
                 gv_smem[(j * GV_COLS + c) * p.kw_pad + d] = v;
                 part += p.corr[j] * __popc(v);
             }
@@ -240,7 +242,7 @@ qnn_status gemv_planes_launch(const qnn_gemm_desc *d, const void *W, const void 
         }
     }
 
-    const size_t smem = (size_t)d->a_bits * GV_COLS * p.kw_pad * 4;
+    const size_t smem = (size_t)d->a_bits * GV_COLS * p.kw_pad * 4;     // [plane][column slot][word]
     const int row_blocks = ceil_div(d->M, GV_THREADS / 32);
     const int max_blocks = sm_count() * 8;
     dim3 grid(row_blocks < max_blocks ? row_blocks : max_blocks, ceil_div(d->N, GV_COLS));
