@@ -33,8 +33,10 @@ __device__ __forceinline__ int dot4(uint32_t w, uint32_t a, int c) {
     return d;
 }
 
+// At most 36 registers, so that 7 CTAs share an SM and the 1024 CTAs of an 8192-row layer are
+// resident in a single wave.
 template <bool W_SIGNED, bool A_SIGNED, int V>
-__global__ void __launch_bounds__(G8_THREADS)
+__global__ void __launch_bounds__(G8_THREADS, 7)
 gemv_i8_kernel(const G8Params p) {
     extern __shared__ __align__(16) uint8_t g8_smem[];     // [G8_COLS][ld] activation bytes
     pdl_wait();
@@ -58,7 +60,7 @@ gemv_i8_kernel(const G8Params p) {
         const uint4 *wrow = reinterpret_cast<const uint4 *>(p.W + (size_t)m * p.ld);
         // a lane takes V consecutive 16-byte units per step (whole sectors; a warp 512 V bytes)
         const int groups = steps / V;
-#pragma unroll 4
+#pragma unroll 2
         for (int q = lane; q < groups; q += 32) {
             uint4 w[V];
 #pragma unroll

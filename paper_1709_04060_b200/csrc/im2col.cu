@@ -35,7 +35,7 @@ struct LowerParams {
     int row_units;              // units per lowered row that are written
     int row_copy;               // KH*KW*cu: units per lowered row that carry data
     long long npix;             // B*OH*OW
-    FastDiv seg, cud, ohow, owd;
+    FastDiv seg, cud, owd;
 };
 
 template <typename T>
@@ -161,7 +161,6 @@ qnn_status im2col_launch(const qnn_conv_desc *d, const void *in, void *lowered, 
     p.npix = (long long)d->B * p.OH * p.OW;
     if (p.OH * p.OW >= 65536 || p.OW >= 65536) return QNN_ERR_UNSUPPORTED;
     p.owd = make_fastdiv(p.OW);
-    p.ohow = make_fastdiv(1);
     const int threads = 256;
     const long long max_blocks = (long long)sm_count() * 16;
 
