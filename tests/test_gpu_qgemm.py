@@ -309,3 +309,43 @@ def test_streamlined_layer_end_to_end(qb):
         torch.cuda.synchronize()
         got = decode_out(out.cpu().numpy(), INT8, 2, 256, 64, False)
         assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("path", [0, 2])
+def test_extreme_operands_and_accumulators(qb, path):
+    """Degenerate and extreme inputs: every operand at the end of its range, so that every
+    accumulator sits at the analytic bound K * max|w| * max|a| (here up to 1.07e9, close to
+    the int32 limit the library accepts), with thresholds at and next to those values."""
+    K = 32768
+    for wv, av in ((-128, 255), (127, 255), (-128, 0)):
+        W = np.full((130, K), wv, dtype=np.int32)
+        W[7] = 0; W[8, ::2] = -wv - 1 if wv < 0 else -wv          # a zero row and a mixed row
+        At = np.full((70, K), av, dtype=np.int32)
+        At[3] = 0; At[4, : K // 2] = 1
+        acc = int(wv) * int(av) * K
+        thr = np.sort(np.array([[acc - 1, acc, acc + 1, 0, -1, 1, 2**31 - 1]] * 130, dtype=np.int64), axis=1)
+        thr = np.clip(thr, -2**31, 2**31 - 1).astype(np.int32)
+        case = synth.GemmCase(130, 70, K, 8, 8, synth.SIGNED, synth.UNSIGNED, 3, W, At, thr)
+        run_case(qb, case, INT8, INT8, path=path)
+        run_case(qb, case, INT8, INT8, raw=True, path=path)
+    # few-bit containers and bit planes at their extremes (W4A4: -8 x 15)
+    W = np.full((100, 8192), -8, dtype=np.int32); W[::3] = 7
+    At = np.full((40, 8192), 15, dtype=np.int32); At[::5] = 0
+    thr = np.sort(np.random.default_rng(9).integers(-983040, 983041, size=(100, 15)), axis=1).astype(np.int32)
+    thr[0] = -983040; thr[1] = 983040 - 122880                   # exactly the extreme accumulators
+    case = synth.GemmCase(100, 40, 8192, 4, 4, synth.SIGNED, synth.UNSIGNED, 4, W, At, thr)
+    run_case(qb, case, INT8, INT8, path=path)
+    if path == 0:
+        run_case(qb, case, BITPLANES, INT8)
+        run_case(qb, case, BITPLANES, BITPLANES)
+
+
+def test_accumulator_range_is_checked_on_the_host(qb):
+    """K * max|w| * max|a| >= 2^31 cannot be accumulated in int32: refused before any launch."""
+    K = 65808                                   # 65808 * 128 * 255 = 2^31 + 489472
+    d = qb.gemm_desc(64, 64, K, 8, 8, 2, qb.QNN_ENC_SIGNED, qb.QNN_ENC_UNSIGNED, INT8, INT8)
+    buf = torch.zeros(64 * K, dtype=torch.uint8, device="cuda")
+    out = torch.zeros(64 * 64, dtype=torch.uint8, device="cuda")
+    n0 = qb.qnn_launch_count()
+    assert qb.qnn_qgemm(d, buf, buf, None, out) == qb.QNN_ERR_UNSUPPORTED
+    assert qb.qnn_launch_count() == n0
