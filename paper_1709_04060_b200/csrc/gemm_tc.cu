@@ -58,9 +58,12 @@ __device__ long long g_trace[16 * 512];
 __device__ int g_trace_cta;
 #define QNN_TRACE(slot, idx) do { if (blockIdx.x == g_trace_cta && (idx) < 512) g_trace[(slot) * 512 + (idx)] = clock64(); } while (0)
 #define QNN_TRACE_NS(idx) do { if (blockIdx.x == g_trace_cta) { long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_trace[8 * 512 + (idx)] = t_; } } while (0)
+// per-CTA wall-clock stamp (slot indexed by CTA): shows how evenly the CTAs finish
+#define QNN_TRACE_CTA(slot) do { if (threadIdx.x == 0 && blockIdx.x < 512) { long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_trace[(slot) * 512 + blockIdx.x] = t_; } } while (0)
 #else
 #define QNN_TRACE(slot, idx) do { } while (0)
 #define QNN_TRACE_NS(idx) do { } while (0)
+#define QNN_TRACE_CTA(slot) do { } while (0)
 #endif
 
 constexpr int TC_BP = 128;          // activation rows (pixels) per tile = tensor-memory lanes
@@ -647,6 +650,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint32_t tmem_base = sm.tmem_base;
     if (threadIdx.x == 0) QNN_TRACE(4, 1);
+    QNN_TRACE_CTA(10);
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
@@ -665,7 +669,9 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
                 for (int kb = un.kb0; kb < un.kb1; ++kb, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1;
+                    QNN_TRACE(14, it);
                     if (!(ok = mbar_wait(&sm.empty[s], ph ^ 1, abort_flag))) break;
+                    QNN_TRACE(15, it);
                     mbar_arrive_expect_tx(&sm.full[s], STAGE_BYTES);
                     if (p.taps) {
                         const int tap = kb / p.cchunks, cc = kb - tap * p.cchunks;
@@ -701,8 +707,10 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
                 for (int kb = un.kb0; kb < un.kb1; ++kb, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1;
+                    QNN_TRACE(12, it);
                     if (!(ok = mbar_wait(&sm.full[s], ph, abort_flag))) break;
                     tc_fence_after();
+                    QNN_TRACE(13, it);
                     if (kb == un.kb0) QNN_TRACE(6, tcount);
                     const uint64_t da = umma_smem_desc(smem_u32(sm.act[s]));
                     const uint64_t db = umma_smem_desc(smem_u32(sm.wgt[s]));
@@ -755,6 +763,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
     if (p.share) cluster_sync_all();       // the peer may still write this CTA's shared memory or barriers
     else __syncthreads();
     if (threadIdx.x == 0) { QNN_TRACE(4, 2); QNN_TRACE_NS(2); }
+    QNN_TRACE_CTA(11);
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);

@@ -85,15 +85,22 @@ __global__ void __launch_bounds__(256) lower_units_kernel(const LowerParams p) {
 // 16-byte read is five aligned words and four funnel shifts.
 constexpr int LR_PIX = 64;
 
+// Bytes of one staged input-row segment in shared memory: the segment may start up to three
+// bytes into its first word (whole aligned words are staged).
+__host__ __device__ inline int lr_seg_pitch(int span, int cu) { return (span * cu + 3 + 3) & ~3; }
+__host__ __device__ inline int lr_head_bytes(int KH) { return (KH * 4 + 15) & ~15; }
+
 __global__ void __launch_bounds__(256) lower_runs_kernel(const LowerParams p, int chunks, int span, int run,
-                                                         int runp) {
-    extern __shared__ __align__(16) uint8_t lr_smem[];   // [KH][seg_pitch] + slack
+                                                         int runp, FastDiv vecd) {
+    extern __shared__ __align__(16) uint8_t lr_smem[];   // [KH] first-byte offsets, [KH][seg_pitch], slack
     pdl_enter();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint8_t *in = reinterpret_cast<const uint8_t *>(p.in);
-    const uint32_t *sm_words = reinterpret_cast<const uint32_t *>(lr_smem);
+    int *seg_off = reinterpret_cast<int *>(lr_smem);
+    uint8_t *segs = lr_smem + lr_head_bytes(p.KH);
+    uint32_t *seg_words = reinterpret_cast<uint32_t *>(segs);
     const int seg_bytes = span * p.cu;                   // bytes of one staged input-row segment
-    const int seg_pitch = (seg_bytes + 3) & ~3;
+    const int seg_pitch = lr_seg_pitch(span, p.cu);
     const int vecs = runp >> 4;                          // 16-byte stores per run
     const long long jobs = (long long)p.B * p.OH * chunks;
     for (long long job = blockIdx.x; job < jobs; job += gridDim.x) {
@@ -104,19 +111,36 @@ __global__ void __launch_bounds__(256) lower_runs_kernel(const LowerParams p, in
         const int npx = min(LR_PIX, p.OW - ow0);
         const int ih0 = oh * p.stride - p.pad, iw0 = ow0 * p.stride - p.pad;
         __syncthreads();                                 // previous job's readers are done
-        // stage: one warp per filter row, lanes along the bytes of the segment
+        // stage: one warp per filter row, lanes along the segment
         for (int kh = warp; kh < p.KH; kh += 8) {
             const int ih = ih0 + kh;
             const bool row_ok = ih >= 0 && ih < p.H;
-            const uint8_t *row = in + (((size_t)b * p.H + (row_ok ? ih : 0)) * p.W) * p.pitch;
-            uint8_t *dst = lr_smem + kh * seg_pitch;
             if (p.pitch == p.cu) {
-                // pixels are contiguous: byte r of the segment is byte iw0*C + r of the image row
-                const int lo = max(0, -iw0) * p.cu, hi = min(span, p.W - iw0) * p.cu;
-                const uint8_t *src = row + (long long)iw0 * p.cu;
-                for (int r = lane; r < seg_pitch; r += 32)
-                    dst[r] = (row_ok && r >= lo && r < hi) ? src[r] : (uint8_t)0;
+                // pixels are contiguous: the segment is bytes [off, off + seg_bytes) of the map.
+                // Whole aligned words are copied (the segment then starts `a` bytes into its
+                // first word); words that straddle the image row's ends are built from bytes.
+                const long long off = (((long long)b * p.H + (row_ok ? ih : 0)) * p.W + iw0) * p.cu;
+                const int a = row_ok ? (int)(off & 3) : 0;
+                const int lo = row_ok ? max(0, -iw0) * p.cu : 0, hi = row_ok ? min(span, p.W - iw0) * p.cu : 0;
+                const uint8_t *base = in + (off - a);
+                uint32_t *dst = seg_words + kh * (seg_pitch >> 2);
+                if (lane == 0) seg_off[kh] = a;
+                for (int r = lane; r < (seg_pitch >> 2); r += 32) {
+                    const int q0 = 4 * r - a;            // segment-relative index of the word's first byte
+                    uint32_t w = 0;
+                    if (q0 >= lo && q0 + 4 <= hi) {
+                        w = *reinterpret_cast<const uint32_t *>(base + 4 * r);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            if (q0 + j >= lo && q0 + j < hi) w |= (uint32_t)base[4 * r + j] << (8 * j);
+                    }
+                    dst[r] = w;
+                }
             } else {
+                const uint8_t *row = in + (((size_t)b * p.H + (row_ok ? ih : 0)) * p.W) * p.pitch;
+                uint8_t *dst = segs + kh * seg_pitch;
+                if (lane == 0) seg_off[kh] = 0;
                 for (int r = lane; r < seg_pitch; r += 32) {
                     const int px = (int)fdiv((uint32_t)r, p.cud), c = r - px * p.cu;
                     const int iw = iw0 + px;
@@ -126,28 +150,29 @@ __global__ void __launch_bounds__(256) lower_runs_kernel(const LowerParams p, in
             }
         }
         __syncthreads();
+        // one 16-byte store per item; item = (pixel, filter row, 16-byte piece of the run), which is
+        // also the order of the output, so a warp writes 512 consecutive bytes
         uint4 *out_row = reinterpret_cast<uint4 *>(p.out) +
                          (((size_t)b * p.OH + oh) * p.OW + ow0) * (size_t)(p.KH * vecs);
-        for (int task = threadIdx.x; task < npx * p.KH; task += blockDim.x) {
+        const int items = npx * p.KH * vecs;
+        for (int item = threadIdx.x; item < items; item += blockDim.x) {
+            const int task = (int)fdiv((uint32_t)item, vecd), v = item - task * vecs;
             const int px = (int)fdiv((uint32_t)task, p.seg), kh = task - px * p.KH;    // p.seg divides by KH here
-            const int src = kh * seg_pitch + px * p.stride * p.cu;
+            const int src = kh * seg_pitch + seg_off[kh] + px * p.stride * p.cu + 16 * v;
             const int sh = (src & 3) * 8;
-            const uint32_t *w = sm_words + (src >> 2);
-            uint4 *dst = out_row + (size_t)task * vecs;
-            for (int v = 0; v < vecs; ++v) {
-                uint32_t x[5];
+            const uint32_t *w = seg_words + (src >> 2);
+            uint32_t x[5];
 #pragma unroll
-                for (int i = 0; i < 5; ++i) x[i] = w[4 * v + i];
-                uint32_t o[4];
+            for (int i = 0; i < 5; ++i) x[i] = w[i];
+            uint32_t o[4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    o[i] = __funnelshift_r(x[i], x[i + 1], sh);
-                    const int valid = run - (16 * v + 4 * i);          // bytes of this word inside the run
-                    if (valid <= 0) o[i] = 0;
-                    else if (valid < 4) o[i] &= (1u << (8 * valid)) - 1u;
-                }
-                dst[v] = make_uint4(o[0], o[1], o[2], o[3]);
+            for (int i = 0; i < 4; ++i) {
+                o[i] = __funnelshift_r(x[i], x[i + 1], sh);
+                const int valid = run - (16 * v + 4 * i);              // bytes of this word inside the run
+                if (valid <= 0) o[i] = 0;
+                else if (valid < 4) o[i] &= (1u << (8 * valid)) - 1u;
             }
+            out_row[item] = make_uint4(o[0], o[1], o[2], o[3]);
         }
     }
 }
@@ -192,13 +217,13 @@ qnn_status im2col_launch(const qnn_conv_desc *d, const void *in, void *lowered, 
 
     if (mode == 2) {
         const int span = (LR_PIX - 1) * d->stride + d->KW;
-        const size_t smem = (size_t)d->KH * ((span * p.cu + 3) & ~3) + 32;      // slack: reads run past a segment
-        if (smem > 48 * 1024 || LR_PIX * d->KH >= 65536) return QNN_ERR_UNSUPPORTED;
+        const size_t smem = (size_t)lr_head_bytes(d->KH) + (size_t)d->KH * lr_seg_pitch(span, p.cu) + 32;   // slack: reads run past a segment
+        if (smem > 48 * 1024 || LR_PIX * d->KH * (runp >> 4) >= 65536) return QNN_ERR_UNSUPPORTED;
         p.seg = make_fastdiv(d->KH);
         const int chunks = ceil_div(p.OW, LR_PIX);
         long long nb = (long long)d->B * p.OH * chunks;
         if (nb > max_blocks) nb = max_blocks;
-        lower_runs_kernel<<<(unsigned)nb, threads, smem, s>>>(p, chunks, span, run, runp);
+        lower_runs_kernel<<<(unsigned)nb, threads, smem, s>>>(p, chunks, span, run, runp, make_fastdiv(runp >> 4));
         count_launch();
         return launch_status();
     }
