@@ -223,6 +223,9 @@ qnn_status qnn_qconv(const qnn_conv_desc *d, const void *Wpacked, const void *in
     if (path == QNN_PATH_TCGEN05_I8 && !(explicit_env && explicit_env[0] == '1')) {
         st = gemm_tc_conv_launch(d, &g, Wpacked, in, thr, out, (cudaStream_t)stream);
         if (st != QNN_ERR_UNSUPPORTED) return st;
+        // few channels, contiguous pixels (the first layer): lowering warps inside the kernel
+        st = gemm_tc_lower_launch(d, &g, Wpacked, in, thr, out, (cudaStream_t)stream);
+        if (st != QNN_ERR_UNSUPPORTED) return st;
     }
     st = im2col_launch(d, in, workspace, (cudaStream_t)stream);
     if (st != QNN_OK) return st;

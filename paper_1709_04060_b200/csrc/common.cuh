@@ -61,6 +61,8 @@ qnn_status gemm_tc_launch(const qnn_gemm_desc *d, const void *W, const void *A,
                           const int32_t *thr, void *out, cudaStream_t s);
 qnn_status gemm_tc_conv_launch(const qnn_conv_desc *cv, const qnn_gemm_desc *g, const void *W, const void *in,
                                const int32_t *thr, void *out, cudaStream_t s);
+qnn_status gemm_tc_lower_launch(const qnn_conv_desc *cv, const qnn_gemm_desc *g, const void *W, const void *in,
+                                const int32_t *thr, void *out, cudaStream_t s);
 qnn_status im2col_launch(const qnn_conv_desc *d, const void *in, void *lowered, cudaStream_t s);
 qnn_status maxpool_launch(const qnn_pool_desc *d, const void *in, void *out, cudaStream_t s);
 qnn_status validate_thresholds_launch(const int32_t *thr, int M, int n_thr, int *n_bad, cudaStream_t s);

@@ -84,13 +84,16 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t by
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
                  : "memory");
 }
+// One try: the thread is suspended until the phase completes or the time hint runs out (it
+// issues nothing meanwhile, so waiting roles leave the issue slots to the working ones).
+constexpr uint32_t MBAR_SUSPEND_NS = 20000;
 __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.b32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(MBAR_SUSPEND_NS) : "memory");
     return ok != 0;
 }
 // Bounded wait.  Returns false if the limit ran out or another role gave up.
@@ -132,9 +135,9 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity
         uint32_t ok;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
             "selp.b32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+            : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(MBAR_SUSPEND_NS) : "memory");
         if (ok) return true;
         if (*abort_flag) return false;
         if (clock64() - t0 > TC_WAIT_CYCLES) {
@@ -209,7 +212,30 @@ struct TcParams {
     // channels-last feature map itself: k-block kb = (filter tap, 128-byte channel chunk), and
     // the 128 pixels x 128 bytes of a stage are fetched by one im2col-mode TMA load.
     int taps, cchunks, cv_C, cv_KW, cv_OW, cv_OHW, cv_stride, cv_pad;
+    // Convolution lowered inside the kernel (LOWER kernels; 8-bit maps with contiguous pixels whose
+    // channel count is not a multiple of 16, no padding): the map itself is the input, four
+    // lowering warps build the activation tiles of the run-per-filter-row lowering in shared
+    // memory from image rows staged there by bulk copies.
+    const uint8_t *lw_in;  // the map [B][H][W][C]
+    long long lw_total;    // its size in bytes
+    int lw_H, lw_KH;       // image rows, filter rows
+    int lw_rowbytes;       // W*C: bytes of an image row
+    int lw_step;           // stride*C: bytes between the runs of neighbouring output pixels
+    int lw_run, lw_vecs;   // bytes of a run (KW*C) and its 16-byte pieces
+    int lw_stage_bytes;    // bytes of one staging buffer
 };
+
+constexpr int LW_WARPS = 4;                    // lowering warps of the LOWER kernels
+constexpr int LW_THREADS = 32 * LW_WARPS;      // = TC_BP: one thread per pixel of the tile
+
+// Byte range [lo, hi) of the map that the runs of output pixels [p0, p1] touch (whole image rows),
+// lo rounded down to 16.
+__host__ __device__ inline void lw_range(const TcParams &p, int p0, int p1, long long *lo, long long *hi) {
+    const int b0 = p0 / p.cv_OHW, oh0 = (p0 - b0 * p.cv_OHW) / p.cv_OW;
+    const int b1 = p1 / p.cv_OHW, oh1 = (p1 - b1 * p.cv_OHW) / p.cv_OW;
+    *lo = (((long long)b0 * p.lw_H + (long long)oh0 * p.cv_stride) * p.lw_rowbytes) & ~15ll;
+    *hi = ((long long)b1 * p.lw_H + (long long)oh1 * p.cv_stride + p.lw_KH) * p.lw_rowbytes;
+}
 
 // What an epilogue warp needs for the exchange of a shared tile.  The weight ring holds,
 // per lane quarter q, a landing slab (what the peer sends) and a staging slab (what this
@@ -610,17 +636,22 @@ struct TcSmem {
     uint64_t thr_empty[2];
     uint64_t ring_free;
     uint64_t landed[4 * 4];
+    uint64_t w_full;           // LOWER: the resident weights have landed
+    uint64_t in_full[2];       // LOWER: image rows of a unit have landed in staging buffer b
+    uint64_t in_empty[2];      // LOWER: the lowering warps are done with staging buffer b
     uint32_t tmem_base;
     int abort_flag;
 };
 
-template <int BN, int STAGES, int OUT_MODE, int OUT_BITS>
-__global__ void __launch_bounds__(TC_THREADS, 1)
+template <int BN, int STAGES, int OUT_MODE, int OUT_BITS, int LOWER>
+__global__ void __launch_bounds__(LOWER ? TC_THREADS + LW_THREADS : TC_THREADS, 1)
 qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_constant__ CUtensorMap map_wgt,
                 const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
     using Smem = TcSmem<BN, STAGES, OUT_BITS>;
-    Smem &sm = *reinterpret_cast<Smem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    // 1024-byte alignment by an offset into the array (not by rounding the pointer's integer
+    // value), so that the compiler still knows these are shared-memory addresses
+    Smem &sm = *reinterpret_cast<Smem *>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u));
     constexpr uint32_t TMEM_COLS = (2 * BN < 32) ? 32 : 2 * BN;
     constexpr uint32_t STAGE_BYTES = (TC_BP + BN) * TC_BK;
 
@@ -629,11 +660,14 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
     if (threadIdx.x == 0) { QNN_TRACE(4, 0); QNN_TRACE_NS(0); }
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
+        // LOWER: a stage is full when every lowering thread has written its row of the activation tile
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&sm.full[s], LOWER ? LW_THREADS : 1); mbar_init(&sm.empty[s], 1); }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&sm.tmem_full[b], 1); mbar_init(&sm.tmem_empty[b], EPI_WARPS);
             mbar_init(&sm.thr_full[b], 1); mbar_init(&sm.thr_empty[b], EPI_WARPS);
+            mbar_init(&sm.in_full[b], 1); mbar_init(&sm.in_empty[b], LW_WARPS);
         }
+        mbar_init(&sm.w_full, 1);
         mbar_init(&sm.ring_free, 1);
         for (int e = 0; e < 16; ++e) mbar_init(&sm.landed[e], 1);
         sm.abort_flag = 0;
@@ -652,7 +686,117 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
     if (threadIdx.x == 0) QNN_TRACE(4, 1);
     QNN_TRACE_CTA(10);
 
-    if (warp == 0) {
+    // LOWER kernels: after the struct come weight k-blocks STAGES.. (k-blocks 0..STAGES-1 live in the
+    // weight ring, which these kernels do not cycle: the whole weight matrix stays resident) and
+    // the two staging buffers for image rows.
+    uint8_t *const w_extra = reinterpret_cast<uint8_t *>(&sm) + ((sizeof(Smem) + 1023) & ~size_t(1023));
+    uint8_t *const stage_in = w_extra + (LOWER && p.num_kb > STAGES ? (size_t)(p.num_kb - STAGES) * BN * TC_BK : 0);
+    auto w_block = [&](int kb) -> uint8_t * { return kb < STAGES ? sm.wgt[kb] : w_extra + (size_t)(kb - STAGES) * BN * TC_BK; };
+    if (LOWER && warp == 0) {
+        // ------------------- producer of the LOWER kernels: the weights once, then image rows
+        if (lane == 0) {
+            mbar_arrive_expect_tx(&sm.w_full, (uint32_t)p.num_kb * BN * TC_BK);
+            for (int kb = 0; kb < p.num_kb; ++kb) tma_load_2d(w_block(kb), &map_wgt, &sm.w_full, kb * TC_BK, 0);
+            uint32_t n = 0;                                    // the unit's index in this CTA
+            bool ok = true;
+            for (int u = blockIdx.x; ok && u < p.units; u += gridDim.x, ++n) {
+                // image rows of unit u into staging buffer n & 1
+                const uint32_t ib = n & 1;
+                if (!(ok = mbar_wait(&sm.in_empty[ib], ((n >> 1) & 1) ^ 1, abort_flag))) break;
+                const TcUnit un = tc_unit(p, u, BN);
+                long long lo, hi;
+                lw_range(p, un.p0, min(un.p0 + TC_BP, p.N) - 1, &lo, &hi);
+                uint8_t *dst = stage_in + (size_t)ib * p.lw_stage_bytes;
+                // whole 16-byte units by one bulk copy; the copy stays inside the map, whose last
+                // (fewer than 16) bytes are fetched by plain loads when the unit reaches them
+                long long end = (hi + 15) & ~15ll;
+                if (end > p.lw_total) {
+                    end = p.lw_total & ~15ll;
+                    for (long long q = end; q < p.lw_total; ++q) dst[q - lo] = p.lw_in[q];
+                }
+                const uint32_t bytes = (uint32_t)(end - lo);
+                mbar_arrive_expect_tx(&sm.in_full[ib], bytes);
+                asm volatile(
+                    "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                    ::"r"(smem_u32(dst)), "l"(p.lw_in + lo), "r"(bytes), "r"(smem_u32(&sm.in_full[ib])) : "memory");
+            }
+            // gave up: let the copies issued last land before the CTA exits
+            if (!ok) {
+                mbar_wait(&sm.w_full, 0, abort_flag);
+                if (n > 0) mbar_wait(&sm.in_full[(n - 1) & 1], ((n - 1) >> 1) & 1, abort_flag);
+            }
+        }
+        __syncwarp();
+    } else if (LOWER && warp > STAGER_WARP) {
+        // ------------------------------------------------------------ lowering warps
+        // Thread t builds row t of every activation tile: the 128 depth bytes of pixel p0 + t in
+        // k-block kb are pieces 8*kb .. 8*kb+7 of its lowered row (piece V = 16 bytes of run
+        // V / vecs at offset 16 * (V % vecs); a run is contiguous in the staged image row).  The
+        // tile has the layout a 128-byte-swizzled tensor-map copy would give it: 16-byte piece c
+        // of row r sits at piece position c ^ (r & 7).
+        const int t = threadIdx.x - 32 * (STAGER_WARP + 1);
+        uint32_t it = 0, ucount = 0;
+        const int total_vecs = p.lw_KH * p.lw_vecs;
+        uint32_t m_last[4];                                   // byte masks of a run's last piece
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int valid = p.lw_run - (16 * (p.lw_vecs - 1) + 4 * i);
+            m_last[i] = valid >= 4 ? 0xffffffffu : (valid <= 0 ? 0u : (1u << (8 * valid)) - 1u);
+        }
+        for (int u = blockIdx.x; u < p.units; u += gridDim.x, ++ucount) {
+            const TcUnit un = tc_unit(p, u, BN);
+            const uint32_t ib = ucount & 1;
+            const int pix = min(un.p0 + t, p.N - 1);
+            const int b = pix / p.cv_OHW, r = pix - b * p.cv_OHW, oh = r / p.cv_OW, ow = r - oh * p.cv_OW;
+            long long lo, hi;
+            lw_range(p, un.p0, min(un.p0 + TC_BP, p.N) - 1, &lo, &hi);
+            const int off = (int)((((long long)b * p.lw_H + (long long)oh * p.cv_stride) * p.lw_rowbytes +
+                                   (long long)ow * p.lw_step) - lo);
+            const int src_px = (int)ib * p.lw_stage_bytes + off;        // byte offset of this pixel's first run in stage_in
+            if (!warp_wait(&sm.in_full[ib], (ucount >> 1) & 1, lane, abort_flag)) break;
+            // Piece V = 8 * kb + c of the lowered row is piece v of run kh; `so` is its byte offset in
+            // stage_in.  Branch-free (selects only), so that the eight pieces of a k-block form one
+            // block of independent loads and shifts.
+            int v = 0, so = src_px, vleft = total_vecs;
+            bool ok = true;
+            for (int kb = un.kb0; kb < un.kb1; ++kb, ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (it / STAGES) & 1;
+                if (!(ok = warp_wait(&sm.empty[s], ph ^ 1, lane, abort_flag))) break;
+                const uint32_t row = (smem_u32(sm.act[s]) + (uint32_t)t * TC_BK) ^ (uint32_t)((t & 7) << 4);
+                uint32_t o[TC_BK / 16][4];
+#pragma unroll
+                for (int c = 0; c < TC_BK / 16; ++c) {
+                    const bool live = c < vleft, last = v == p.lw_vecs - 1;
+                    // an unaligned 16-byte read: five aligned words and four funnel shifts
+                    const int a = live ? so : src_px;
+                    const uint32_t *w = reinterpret_cast<const uint32_t *>(stage_in) + (a >> 2);
+                    const int sh = (a & 3) * 8;
+                    uint32_t x[5];
+#pragma unroll
+                    for (int i = 0; i < 5; ++i) x[i] = w[i];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const uint32_t m = live ? (last ? m_last[i] : 0xffffffffu) : 0u;
+                        o[c][i] = __funnelshift_r(x[i], x[i + 1], sh) & m;
+                    }
+                    so += last ? p.lw_rowbytes - 16 * (p.lw_vecs - 1) : 16;
+                    v = last ? 0 : v + 1;
+                }
+                vleft -= TC_BK / 16;
+#pragma unroll
+                for (int c = 0; c < TC_BK / 16; ++c)
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                                 ::"r"(row ^ (uint32_t)(c << 4)), "r"(o[c][0]), "r"(o[c][1]), "r"(o[c][2]), "r"(o[c][3])
+                                 : "memory");
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // visible to the tensor core's reads
+                mbar_arrive(&sm.full[s]);
+            }
+            if (!ok) break;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.in_empty[ib]);
+        }
+    } else if (warp == 0) {
         // ------------------------------------------------------------ producer
         if (lane == 0) {
             uint32_t it = 0;
@@ -697,6 +841,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
         if (lane == 0) {
             uint32_t it = 0, tcount = 0;
             bool ok = true;
+            if (LOWER) ok = mbar_wait(&sm.w_full, 0, abort_flag);
             for (int u = blockIdx.x; ok && u < p.units; u += gridDim.x, ++tcount) {
                 const uint32_t buf = tcount & 1, acc_ph = (tcount >> 1) & 1;
                 const TcUnit un = tc_unit(p, u, BN);
@@ -713,11 +858,15 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
                     QNN_TRACE(13, it);
                     if (kb == un.kb0) QNN_TRACE(6, tcount);
                     const uint64_t da = umma_smem_desc(smem_u32(sm.act[s]));
-                    const uint64_t db = umma_smem_desc(smem_u32(sm.wgt[s]));
+                    const uint64_t db = umma_smem_desc(smem_u32(LOWER ? w_block(kb) : sm.wgt[s]));
                     // a channel chunk may hold fewer than 128 real bytes: skip the all-zero MMAs
                     int nk = TC_BK / 32;
                     if (p.taps) {
                         const int left = p.cv_C - (kb % p.cchunks) * TC_BK;
+                        if (left < TC_BK) nk = (left + 31) >> 5;
+                    }
+                    if (LOWER) {
+                        const int left = p.K - kb * TC_BK;
                         if (left < TC_BK) nk = (left + 31) >> 5;
                     }
 #pragma unroll
@@ -829,7 +978,9 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_const
                  const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
     using Smem = Tc2Smem<OUT_BITS>;
-    Smem &sm = *reinterpret_cast<Smem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    // 1024-byte alignment by an offset into the array (not by rounding the pointer's integer
+    // value), so that the compiler still knows these are shared-memory addresses
+    Smem &sm = *reinterpret_cast<Smem *>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u));
     constexpr uint32_t TMEM_COLS = 2 * T2_BN;
     constexpr uint32_t PAIR_STAGE_BYTES = 2 * (TC_BP + 128) * TC_BK;   // both CTAs' copies of one stage
 
@@ -1002,19 +1153,29 @@ static bool make_im2col_map(CUtensorMap *map, const void *base, const qnn_conv_d
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, int STAGES, int OUT_MODE, int OUT_BITS>
+// Shared memory of a LOWER kernel besides its two staging buffers.
+template <int BN, int STAGES, int OUT_BITS>
+constexpr size_t tc_lower_base_smem() { return ((sizeof(TcSmem<BN, STAGES, OUT_BITS>) + 1023) & ~size_t(1023)) + 1024; }
+constexpr size_t TC_SMEM_LIMIT = 227 * 1024;
+
+template <int BN, int STAGES, int OUT_MODE, int OUT_BITS, int LOWER = 0>
 static qnn_status launch_cfg(const CUtensorMap &ma, const CUtensorMap &mw, const TcParams &p, cudaStream_t s) {
-    auto kern = qgemm_tc_kernel<BN, STAGES, OUT_MODE, OUT_BITS>;
-    const size_t smem = sizeof(TcSmem<BN, STAGES, OUT_BITS>) + 1024;
-    static bool attr_done = false;        // per instantiation
-    if (!attr_done) {
+    auto kern = qgemm_tc_kernel<BN, STAGES, OUT_MODE, OUT_BITS, LOWER>;
+    size_t smem = sizeof(TcSmem<BN, STAGES, OUT_BITS>) + 1024;
+    if (LOWER) {
+        smem = tc_lower_base_smem<BN, STAGES, OUT_BITS>() + 2 * (size_t)p.lw_stage_bytes +
+               (p.num_kb > STAGES ? (size_t)(p.num_kb - STAGES) * BN * TC_BK : 0);
+        if (smem > TC_SMEM_LIMIT) return QNN_ERR_UNSUPPORTED;
+    }
+    static size_t attr_smem = 0;          // per instantiation: the largest size configured so far
+    if (smem > attr_smem) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return QNN_ERR_CUDA;
-        attr_done = true;
+        attr_smem = smem;
     }
     const int grid = p.units < sm_count() ? p.units : sm_count();
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(TC_THREADS);
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(LOWER ? TC_THREADS + LW_THREADS : TC_THREADS);
     cfg.dynamicSmemBytes = smem; cfg.stream = s;
     cudaLaunchAttribute attr[2];
     int na = 0;
@@ -1067,10 +1228,10 @@ static qnn_status launch_pair_cfg(const CUtensorMap &ma, const CUtensorMap &mw, 
     }                                                                                      \
     return QNN_ERR_UNSUPPORTED;
 
-template <int BN, int STAGES>
+template <int BN, int STAGES, int LOWER = 0>
 static qnn_status launch_out(int mode, int out_bits, const CUtensorMap &ma, const CUtensorMap &mw,
                              const TcParams &p, cudaStream_t s) {
-#define QNN_C1(MODE_, BITS_) launch_cfg<BN, STAGES, MODE_, BITS_>(ma, mw, p, s)
+#define QNN_C1(MODE_, BITS_) launch_cfg<BN, STAGES, MODE_, BITS_, LOWER>(ma, mw, p, s)
     QNN_TC_DISPATCH(QNN_C1(OUT_RAW, 0), QNN_C1)
 #undef QNN_C1
 }
@@ -1233,6 +1394,66 @@ qnn_status gemm_tc_conv_launch(const qnn_conv_desc *cv, const qnn_gemm_desc *g, 
         cv->KH * cv->KW * ceil_div(cv->C, TC_BK) > ceil_div(g->K, TC_BK))
         return QNN_ERR_UNSUPPORTED;
     return tc_launch(g, cv, W, in, thr, out, s);
+}
+
+// Convolution of an 8-bit map whose channel count is not a multiple of 16 (the 3-channel first
+// layer) with the lowering done inside the kernel; weights in the run-per-filter-row layout of
+// qnn_conv_lowered_k.  UNSUPPORTED: padding, a pixel pitch other than C, more than 128 output
+// channels, or weights plus staged image rows that do not fit shared memory -- the caller then
+// lowers explicitly.
+constexpr int LW_BN = 128, LW_STAGES = 4;
+qnn_status gemm_tc_lower_launch(const qnn_conv_desc *cv, const qnn_gemm_desc *g, const void *W, const void *in,
+                                const int32_t *thr, void *out, cudaStream_t s) {
+    const int pitch = cv->in_pitch ? cv->in_pitch : round_up(cv->C, 16);
+    if (cv->fmt != QNN_FMT_INT8 || (cv->C % 16) == 0 || pitch != cv->C || cv->pad != 0) return QNN_ERR_UNSUPPORTED;
+    const int run = cv->KW * cv->C, runp = round_up(run, 16);
+    if (g->K != cv->KH * runp) return QNN_ERR_UNSUPPORTED;
+    const int OH = qnn_conv_out_h(cv), OW = qnn_conv_out_w(cv);
+    if ((long long)g->N * g->K >= (1ll << 40)) return QNN_ERR_UNSUPPORTED;
+
+    TcParams p;
+    p.thr = thr; p.out = out; p.M = g->M; p.N = g->N; p.K = g->K;
+    p.num_kb = ceil_div(g->K, TC_BK);
+    p.ld_out = round_up(g->M, 16);
+    p.kb_half = 0; p.share = 0;
+    p.taps = 0; p.cchunks = 1; p.cv_C = cv->C; p.cv_KW = cv->KW; p.cv_pad = 0;
+    p.cv_stride = cv->stride; p.cv_OW = OW; p.cv_OHW = OH * OW;
+    p.lw_in = reinterpret_cast<const uint8_t *>(in);
+    p.lw_total = (long long)cv->B * cv->H * cv->W * cv->C;
+    p.lw_H = cv->H; p.lw_KH = cv->KH;
+    p.lw_rowbytes = cv->W * cv->C; p.lw_step = cv->stride * cv->C;
+    p.lw_run = run; p.lw_vecs = runp / 16;
+    // Most image rows a tile of TC_BP consecutive output pixels touches: KH rows for its first
+    // output row, plus, per further output row, `stride` rows inside an image or the
+    // H - (OH-1)*stride rows across an image boundary (an upper bound).
+    const int moves = ceil_div(TC_BP - 1, OW);
+    const int images = moves < ceil_div(TC_BP - 1, OH * OW) ? moves : ceil_div(TC_BP - 1, OH * OW);
+    const int cross = cv->H - (OH - 1) * cv->stride > cv->stride ? cv->H - (OH - 1) * cv->stride : cv->stride;
+    const long long rows = cv->KH + (long long)(moves - images) * cv->stride + (long long)images * cross;
+    const long long stage = rows * p.lw_rowbytes + 16 + 48;          // rounding of the start, reads past a run
+    if (stage > (long long)TC_SMEM_LIMIT) return QNN_ERR_UNSUPPORTED;
+    p.lw_stage_bytes = (int)round_up((int)stage, 128);
+    // the whole weight matrix stays in shared memory: one channel tile, a few k-blocks
+    if (g->M > LW_BN) return QNN_ERR_UNSUPPORTED;
+    const size_t w_extra = p.num_kb > LW_STAGES ? (size_t)(p.num_kb - LW_STAGES) * LW_BN * TC_BK : 0;
+    if (tc_lower_base_smem<LW_BN, LW_STAGES, 4>() + 2 * (size_t)p.lw_stage_bytes + w_extra > TC_SMEM_LIMIT)
+        return QNN_ERR_UNSUPPORTED;
+    p.tiles_p = ceil_div(g->N, TC_BP); p.tiles_c = 1;
+    const long long tiles = (long long)p.tiles_p * p.tiles_c;
+    if (tiles > 0x3fffffff) return QNN_ERR_UNSUPPORTED;
+    p.units = p.full_units = (int)tiles;
+    const double wmax = g->w_enc == QNN_ENC_BIPOLAR ? 1.0
+                        : (g->w_enc == QNN_ENC_SIGNED ? double(1 << (g->w_bits - 1)) : double((1 << g->w_bits) - 1));
+    const double amax = g->a_enc == QNN_ENC_BIPOLAR ? 1.0
+                        : (g->a_enc == QNN_ENC_SIGNED ? double(1 << (g->a_bits - 1)) : double((1 << g->a_bits) - 1));
+    p.fp_count = (double(g->K) * wmax * amax < double(FP_LIMIT)) ? 1 : 0;
+    const uint32_t w_s8 = g->w_enc == QNN_ENC_UNSIGNED ? 0u : 1u;
+    const uint32_t a_s8 = g->a_enc == QNN_ENC_UNSIGNED ? 0u : 1u;
+    p.idesc = (2u << 4) | (a_s8 << 7) | (w_s8 << 10) | ((uint32_t)(LW_BN >> 3) << 17) | ((uint32_t)(TC_BP >> 4) << 24);
+    const int mode = !thr ? OUT_RAW : (g->out_fmt == QNN_FMT_INT8 ? OUT_U8 : OUT_PLANES);
+    CUtensorMap mw;
+    if (!make_map(&mw, W, g->M, g->K, round_up(g->K, 16), LW_BN)) return QNN_ERR_CUDA;
+    return launch_out<LW_BN, LW_STAGES, 1>(mode, g->out_bits, mw, mw, p, s);
 }
 
 #ifdef QNN_TC_TRACE

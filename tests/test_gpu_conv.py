@@ -330,3 +330,46 @@ def test_implicit_convolution_shapes(qb, monkeypatch, shape):
     assert qb.qnn_launch_count() - n0 == 2            # lowering + GEMM
     torch.cuda.synchronize()
     assert torch.equal(raw, raw_explicit)
+
+
+@pytest.mark.parametrize("shape", [
+    # B, H, W, C, OC, KH, KW, stride, pad, w_bits, a_bits
+    (2, 39, 43, 3, 40, 11, 11, 4, 0, 8, 8),       # first-layer filter; map size not a multiple of 16 bytes
+    (3, 227, 227, 3, 96, 11, 11, 4, 0, 8, 8),     # first-layer shape: 71 tiles, tiles across image boundaries
+    (40, 12, 12, 3, 20, 5, 5, 1, 0, 8, 8),        # small images: a tile holds pixels of three images
+    (2, 30, 29, 5, 130, 7, 3, 2, 0, 4, 4),        # more than 128 channels: explicit lowering
+    (2, 30, 29, 5, 128, 7, 3, 2, 0, 4, 4),        # rectangular filter, stride 2, a full channel tile
+    (1, 21, 22, 6, 33, 3, 4, 3, 0, 2, 2),         # stride 3
+    (5, 9, 9, 20, 17, 3, 3, 1, 0, 2, 2),          # 20 channels: runs of 60 bytes in four 16-byte pieces
+    (1, 8, 9, 1, 16, 2, 2, 1, 0, 8, 8),           # one channel, one 16-byte piece per run
+])
+def test_convolution_lowered_inside_the_kernel(qb, monkeypatch, shape):
+    """8-bit maps with contiguous pixels whose channel count is not a multiple of 16, no padding:
+    lowering warps inside the tensor-core kernel build the activation tiles (one launch); against
+    the direct convolution, and the explicit lowering must give the same accumulators."""
+    case = synth.conv_case(1300 + shape[3] + shape[7], *shape, w_enc=synth.SIGNED, a_enc=synth.UNSIGNED)
+    x, pitch = device_map(qb, case, INT8, in_pitch=case.C)
+    Wp = device_weights(qb, case, INT8)
+    npix = case.B * case.OH * case.OW
+    thr = torch.from_numpy(case.thr).cuda()
+    want = orc.qconv(case.In, case.Wt, case.thr, case.stride, case.pad).reshape(npix, case.OC)
+    for out_fmt in (INT8, BITPLANES):
+        d = conv_desc(qb, case, INT8, out_fmt, pitch)
+        n0 = qb.qnn_launch_count()
+        out = qb.qconv(d, Wp, x, thr)
+        # no lowering kernel while the weights fit shared memory (one tile of 128 channels)
+        assert qb.qnn_launch_count() - n0 == (1 if case.OC <= 128 else 2)
+        torch.cuda.synchronize()
+        st, dev = qb.qnn_device_status()
+        assert st == 0 and dev == 0
+        assert np.array_equal(decode_out(out.cpu().numpy(), out_fmt, case.out_bits, npix, case.OC, False), want)
+    d = conv_desc(qb, case, INT8, INT8, pitch)
+    raw = qb.qconv(d, Wp, x, None).clone()
+    monkeypatch.setenv("QNN_CONV_EXPLICIT", "1")
+    n0 = qb.qnn_launch_count()
+    raw_explicit = qb.qconv(d, Wp, x, None)
+    assert qb.qnn_launch_count() - n0 == 2            # lowering + GEMM
+    torch.cuda.synchronize()
+    assert torch.equal(raw, raw_explicit)
+    acc = np.frombuffer(raw.cpu().numpy().tobytes(), dtype=np.int32).reshape(npix, case.OC)
+    assert np.array_equal(acc, orc.conv_direct(case.In, case.Wt, case.stride, case.pad).reshape(npix, case.OC))
