@@ -77,6 +77,7 @@ __device__ __forceinline__ uint32_t container4(uint32_t x, int bits, int enc) {
 __global__ void __launch_bounds__(256) pack_int8_vec_kernel(const uint4 *__restrict__ logical,
                                                             uint4 *__restrict__ packed, long long n16,
                                                             int bits, int enc) {
+    pdl_trigger();        // a tensor-core kernel queued behind the packer may set up while it drains
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n16;
          i += (long long)gridDim.x * blockDim.x) {
         const uint4 v = logical[i];
