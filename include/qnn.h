@@ -174,7 +174,12 @@ qnn_status qnn_im2col(const qnn_conv_desc *d, const void *in, void *lowered, voi
 /* Convolution by lowering + fused GEMM/threshold.  Wpacked: the [OC][K_lowered]
  * weight operand in format d->fmt.  Output: as qnn_qgemm with N = B*OH*OW,
  * M = OC, i.e. a channels-last feature map [B][OH][OW][...].  BIPOLAR
- * activations with pad > 0 are UNSUPPORTED (zero is not representable). */
+ * activations with pad > 0 are UNSUPPORTED (zero is not representable).
+ * The lowered matrix of Section 3.2 is written to `workspace` only where the
+ * GEMM kernel cannot form its tiles itself: 8-bit maps are lowered inside the
+ * kernel (by its tensor-map loader when C and in_pitch are multiples of 16; by
+ * lowering warps when C is not, pixels are contiguous, pad == 0 and OC <= 128),
+ * with the same integer results.  The workspace must be given in every case. */
 qnn_status qnn_qconv(const qnn_conv_desc *d, const void *Wpacked, const void *in,
                      const int32_t *thr, void *out,
                      void *workspace, size_t workspace_bytes, void *stream);
