@@ -179,7 +179,9 @@ qnn_status qnn_im2col(const qnn_conv_desc *d, const void *in, void *lowered, voi
  * GEMM kernel cannot form its tiles itself: 8-bit maps are lowered inside the
  * kernel (by its tensor-map loader when C and in_pitch are multiples of 16; by
  * lowering warps when C is not, pixels are contiguous, pad == 0 and OC <= 128),
- * with the same integer results.  The workspace must be given in every case. */
+ * with the same integer results.  The pad columns of the weight rows (see
+ * qnn_conv_lowered_k) must be zero: the in-kernel lowering leaves image bytes,
+ * not zeros, opposite them.  The workspace must be given in every case. */
 qnn_status qnn_qconv(const qnn_conv_desc *d, const void *Wpacked, const void *in,
                      const int32_t *thr, void *out,
                      void *workspace, size_t workspace_bytes, void *stream);

@@ -737,12 +737,6 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
         const int t = threadIdx.x - 32 * (STAGER_WARP + 1);
         uint32_t it = 0, ucount = 0;
         const int total_vecs = p.lw_KH * p.lw_vecs;
-        uint32_t m_last[4];                                   // byte masks of a run's last piece
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int valid = p.lw_run - (16 * (p.lw_vecs - 1) + 4 * i);
-            m_last[i] = valid >= 4 ? 0xffffffffu : (valid <= 0 ? 0u : (1u << (8 * valid)) - 1u);
-        }
         for (int u = blockIdx.x; u < p.units; u += gridDim.x, ++ucount) {
             const TcUnit un = tc_unit(p, u, BN);
             const uint32_t ib = ucount & 1;
@@ -775,11 +769,12 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
                     uint32_t x[5];
 #pragma unroll
                     for (int i = 0; i < 5; ++i) x[i] = w[i];
+                    // No masking: the bytes past a run's end (and the pieces past the last run) meet
+                    // weight bytes that are zero -- the pad columns of the weight rows, or depth
+                    // positions past K, which the weight copy fills with zeros -- so whatever image
+                    // bytes land there add nothing to the integer sums.
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const uint32_t m = live ? (last ? m_last[i] : 0xffffffffu) : 0u;
-                        o[c][i] = __funnelshift_r(x[i], x[i + 1], sh) & m;
-                    }
+                    for (int i = 0; i < 4; ++i) o[c][i] = __funnelshift_r(x[i], x[i + 1], sh);
                     so += last ? p.lw_rowbytes - 16 * (p.lw_vecs - 1) : 16;
                     v = last ? 0 : v + 1;
                 }
