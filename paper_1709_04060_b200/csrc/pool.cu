@@ -17,8 +17,11 @@ struct PoolParams {
 };
 
 // 16 channels (one uint4) per thread; the padded channel count is a multiple of 16.
+// KT > 0: window size known at compile time (all KT*KT loads of a thread are in flight together).
+template <int KT>
 __global__ void __launch_bounds__(256) maxpool_u8_kernel(const PoolParams p) {
     pdl_enter();
+    const int k = KT > 0 ? KT : p.k;
     const int cu = p.cu >> 2;                                     // 16-byte units per pixel
     const long long total = (long long)p.B * p.OH * p.OW * cu;
     const uint4 *in = reinterpret_cast<const uint4 *>(p.in);
@@ -30,9 +33,11 @@ __global__ void __launch_bounds__(256) maxpool_u8_kernel(const PoolParams p) {
         const unsigned ow = t % (unsigned)p.OW, t2 = t / (unsigned)p.OW;
         const unsigned oh = t2 % (unsigned)p.OH, b = t2 / (unsigned)p.OH;
         uint4 best = make_uint4(0, 0, 0, 0);
-        for (int i = 0; i < p.k; ++i) {
+#pragma unroll
+        for (int i = 0; i < k; ++i) {
             const uint4 *row = in + (((size_t)b * p.H + oh * p.stride + i) * p.W + ow * p.stride) * cu + u;
-            for (int j = 0; j < p.k; ++j) {
+#pragma unroll
+            for (int j = 0; j < k; ++j) {
                 const uint4 v = __ldg(row + (size_t)j * cu);
                 best.x = __vmaxu4(best.x, v.x); best.y = __vmaxu4(best.y, v.y);
                 best.z = __vmaxu4(best.z, v.z); best.w = __vmaxu4(best.w, v.w);
@@ -94,7 +99,9 @@ qnn_status maxpool_launch(const qnn_pool_desc *d, const void *in, void *out, cud
     const long long max_blocks = (long long)sm_count() * 16;
     if (blocks > max_blocks) blocks = max_blocks;
     if (d->fmt == QNN_FMT_INT8) {
-        maxpool_u8_kernel<<<(unsigned)blocks, threads, 0, s>>>(p);
+        if (d->k == 3) maxpool_u8_kernel<3><<<(unsigned)blocks, threads, 0, s>>>(p);
+        else if (d->k == 2) maxpool_u8_kernel<2><<<(unsigned)blocks, threads, 0, s>>>(p);
+        else maxpool_u8_kernel<0><<<(unsigned)blocks, threads, 0, s>>>(p);
     } else {
         switch (d->bits) {
             case 1: maxpool_planes_kernel<1><<<(unsigned)blocks, threads, 0, s>>>(p); break;
