@@ -382,19 +382,21 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams &p, const int *thr
         // distinct banks, so lanes that look at different slots do not conflict
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
-            const int *rows = thr_c + 8 * g * NT;
+            // the search position is carried as a pointer (row + count): every probe is a load at a
+            // constant offset from it, and a step is load, compare, conditional add
+            const int *pos[8];
             int c[8], t[8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) t[e] = rows[e * NT + NT / 2 - 1];
+            for (int e = 0; e < 8; ++e) pos[e] = thr_c + (8 * g + e) * NT;
 #pragma unroll
-            for (int e = 0; e < 8; ++e) c[e] = (acc[8 * g + e] >= t[e]) ? NT / 2 : 0;
+            for (int step = NT / 2; step >= 1; step >>= 1) {
 #pragma unroll
-            for (int step = NT / 4; step >= 1; step >>= 1) {
+                for (int e = 0; e < 8; ++e) t[e] = pos[e][step - 1];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) t[e] = rows[e * NT + c[e] + step - 1];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) c[e] += (acc[8 * g + e] >= t[e]) ? step : 0;
+                for (int e = 0; e < 8; ++e) pos[e] += (acc[8 * g + e] >= t[e]) ? step : 0;
             }
+#pragma unroll
+            for (int e = 0; e < 8; ++e) c[e] = (int)(pos[e] - (thr_c + (8 * g + e) * NT));
             packed[2 * g] = (uint32_t)c[0] | ((uint32_t)c[1] << 8) | ((uint32_t)c[2] << 16) | ((uint32_t)c[3] << 24);
             packed[2 * g + 1] = (uint32_t)c[4] | ((uint32_t)c[5] << 8) | ((uint32_t)c[6] << 16) | ((uint32_t)c[7] << 24);
         }
