@@ -32,6 +32,7 @@
  *   QNN_TC_NO_SHARE=1          never split a tile's depth between two CTAs
  *   QNN_CONV_EXPLICIT=1        qnn_qconv always goes through the lowered matrix
  *   QNN_CONV_IMPLICIT=1        qnn_qconv lowers inside the GEMM wherever it can
+ *   QNN_CONV_LOWER=1           qnn_qconv uses the lowering warps wherever they apply
  *
  * Operand formats
  *   QNN_FMT_BITPLANES  uint32 [bits][rows][kw], kw = ceil(K/32): plane i holds
@@ -178,8 +179,9 @@ qnn_status qnn_im2col(const qnn_conv_desc *d, const void *in, void *lowered, voi
  * The lowered matrix of Section 3.2 is written to `workspace` only where the
  * GEMM kernel cannot form its tiles itself: 8-bit maps are lowered inside the
  * kernel (by its tensor-map loader when C and in_pitch are multiples of 16; by
- * lowering warps when C is not, pixels are contiguous, pad == 0 and OC <= 128),
- * with the same integer results.  The pad columns of the weight rows (see
+ * lowering warps when pixels are contiguous and either C is not a multiple of
+ * 16, pad == 0 and OC <= 128, or C is a multiple of 16 but not of 128 and the
+ * layer has many tiles), with the same integer results.  The pad columns of the weight rows (see
  * qnn_conv_lowered_k) must be zero: the in-kernel lowering leaves image bytes,
  * not zeros, opposite them.  The workspace must be given in every case. */
 qnn_status qnn_qconv(const qnn_conv_desc *d, const void *Wpacked, const void *in,

@@ -221,10 +221,11 @@ qnn_status qnn_qconv(const qnn_conv_desc *d, const void *Wpacked, const void *in
     // lowered matrix (measurements, tests)
     const char *explicit_env = getenv("QNN_CONV_EXPLICIT");
     if (path == QNN_PATH_TCGEN05_I8 && !(explicit_env && explicit_env[0] == '1')) {
-        st = gemm_tc_conv_launch(d, &g, Wpacked, in, thr, out, (cudaStream_t)stream);
-        if (st != QNN_ERR_UNSUPPORTED) return st;
-        // few channels, contiguous pixels (the first layer): lowering warps inside the kernel
+        // lowering warps inside the kernel where the tensor-map loader does not apply (few
+        // channels: the first layer) or would waste k-blocks (channel count not a multiple of 128)
         st = gemm_tc_lower_launch(d, &g, Wpacked, in, thr, out, (cudaStream_t)stream);
+        if (st != QNN_ERR_UNSUPPORTED) return st;
+        st = gemm_tc_conv_launch(d, &g, Wpacked, in, thr, out, (cudaStream_t)stream);
         if (st != QNN_ERR_UNSUPPORTED) return st;
     }
     st = im2col_launch(d, in, workspace, (cudaStream_t)stream);

@@ -212,13 +212,17 @@ struct TcParams {
     // channels-last feature map itself: k-block kb = (filter tap, 128-byte channel chunk), and
     // the 128 pixels x 128 bytes of a stage are fetched by one im2col-mode TMA load.
     int taps, cchunks, cv_C, cv_KW, cv_OW, cv_OHW, cv_stride, cv_pad;
-    // Convolution lowered inside the kernel (LOWER kernels; 8-bit maps with contiguous pixels whose
-    // channel count is not a multiple of 16, no padding): the map itself is the input, four
-    // lowering warps build the activation tiles of the run-per-filter-row lowering in shared
-    // memory from image rows staged there by bulk copies.
+    // Convolution lowered inside the kernel (LOWER kernels; 8-bit maps with contiguous pixels): the
+    // map itself is the input, four lowering warps build the activation tiles in shared memory
+    // from image rows staged there by bulk copies.  A lowered row is one run per filter row: the
+    // KW*C bytes that row contributes, padded to a multiple of 16.  LOWER == 1: C not a multiple
+    // of 16 (unaligned runs), no padding around the image, the whole weight matrix resident in
+    // shared memory.  LOWER == 2: C a multiple of 16 (every 16-byte piece lies in one pixel and is
+    // aligned), zero padding around the image, weights streamed through the ring.
     const uint8_t *lw_in;  // the map [B][H][W][C]
     long long lw_total;    // its size in bytes
     int lw_H, lw_KH;       // image rows, filter rows
+    int lw_W, lw_cpp;      // LOWER == 2: image columns, 16-byte pieces per pixel (C / 16)
     int lw_rowbytes;       // W*C: bytes of an image row
     int lw_step;           // stride*C: bytes between the runs of neighbouring output pixels
     int lw_run, lw_vecs;   // bytes of a run (KW*C) and its 16-byte pieces
@@ -233,8 +237,11 @@ constexpr int LW_THREADS = 32 * LW_WARPS;      // = TC_BP: one thread per pixel 
 __host__ __device__ inline void lw_range(const TcParams &p, int p0, int p1, long long *lo, long long *hi) {
     const int b0 = p0 / p.cv_OHW, oh0 = (p0 - b0 * p.cv_OHW) / p.cv_OW;
     const int b1 = p1 / p.cv_OHW, oh1 = (p1 - b1 * p.cv_OHW) / p.cv_OW;
-    *lo = (((long long)b0 * p.lw_H + (long long)oh0 * p.cv_stride) * p.lw_rowbytes) & ~15ll;
-    *hi = ((long long)b1 * p.lw_H + (long long)oh1 * p.cv_stride + p.lw_KH) * p.lw_rowbytes;
+    int r0 = oh0 * p.cv_stride - p.cv_pad, r1 = oh1 * p.cv_stride - p.cv_pad + p.lw_KH;   // rows of the image
+    if (r0 < 0) r0 = 0;
+    if (r1 > p.lw_H) r1 = p.lw_H;
+    *lo = (((long long)b0 * p.lw_H + r0) * p.lw_rowbytes) & ~15ll;
+    *hi = ((long long)b1 * p.lw_H + r1) * p.lw_rowbytes;
 }
 
 // What an epilogue warp needs for the exchange of a shared tile.  The weight ring holds,
@@ -663,7 +670,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
 
     if (threadIdx.x == 0) {
         // LOWER: a stage is full when every lowering thread has written its row of the activation tile
-        for (int s = 0; s < STAGES; ++s) { mbar_init(&sm.full[s], LOWER ? LW_THREADS : 1); mbar_init(&sm.empty[s], 1); }
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&sm.full[s], LOWER == 1 ? LW_THREADS : (LOWER == 2 ? LW_THREADS + 1 : 1)); mbar_init(&sm.empty[s], 1); }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&sm.tmem_full[b], 1); mbar_init(&sm.tmem_empty[b], EPI_WARPS);
             mbar_init(&sm.thr_full[b], 1); mbar_init(&sm.thr_empty[b], EPI_WARPS);
@@ -692,19 +699,16 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
     // weight ring, which these kernels do not cycle: the whole weight matrix stays resident) and
     // the two staging buffers for image rows.
     uint8_t *const w_extra = reinterpret_cast<uint8_t *>(&sm) + ((sizeof(Smem) + 1023) & ~size_t(1023));
-    uint8_t *const stage_in = w_extra + (LOWER && p.num_kb > STAGES ? (size_t)(p.num_kb - STAGES) * BN * TC_BK : 0);
+    uint8_t *const stage_in = w_extra + (LOWER == 1 && p.num_kb > STAGES ? (size_t)(p.num_kb - STAGES) * BN * TC_BK : 0);
     auto w_block = [&](int kb) -> uint8_t * { return kb < STAGES ? sm.wgt[kb] : w_extra + (size_t)(kb - STAGES) * BN * TC_BK; };
     if (LOWER && warp == 0) {
         // ------------------- producer of the LOWER kernels: the weights once, then image rows
         if (lane == 0) {
-            mbar_arrive_expect_tx(&sm.w_full, (uint32_t)p.num_kb * BN * TC_BK);
-            for (int kb = 0; kb < p.num_kb; ++kb) tma_load_2d(w_block(kb), &map_wgt, &sm.w_full, kb * TC_BK, 0);
-            uint32_t n = 0;                                    // the unit's index in this CTA
-            bool ok = true;
-            for (int u = blockIdx.x; ok && u < p.units; u += gridDim.x, ++n) {
-                // image rows of unit u into staging buffer n & 1
+            uint32_t staged = 0;                               // staging copies issued
+            // image rows of unit u into staging buffer n & 1 (n = the unit's index in this CTA)
+            auto stage_rows = [&](int u, uint32_t n) -> bool {
                 const uint32_t ib = n & 1;
-                if (!(ok = mbar_wait(&sm.in_empty[ib], ((n >> 1) & 1) ^ 1, abort_flag))) break;
+                if (!mbar_wait(&sm.in_empty[ib], ((n >> 1) & 1) ^ 1, abort_flag)) return false;
                 const TcUnit un = tc_unit(p, u, BN);
                 long long lo, hi;
                 lw_range(p, un.p0, min(un.p0 + TC_BP, p.N) - 1, &lo, &hi);
@@ -721,11 +725,35 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
                 asm volatile(
                     "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                     ::"r"(smem_u32(dst)), "l"(p.lw_in + lo), "r"(bytes), "r"(smem_u32(&sm.in_full[ib])) : "memory");
+                staged = n + 1;
+                return true;
+            };
+            bool ok = true;
+            uint32_t n = 0, it = 0;
+            if (LOWER == 1) {
+                // the whole weight matrix once, then nothing but image rows
+                mbar_arrive_expect_tx(&sm.w_full, (uint32_t)p.num_kb * BN * TC_BK);
+                for (int kb = 0; kb < p.num_kb; ++kb) tma_load_2d(w_block(kb), &map_wgt, &sm.w_full, kb * TC_BK, 0);
+                for (int u = blockIdx.x; ok && u < p.units; u += gridDim.x, ++n) ok = stage_rows(u, n);
+            } else {
+                // image rows one unit ahead, weights k-block by k-block through the ring
+                if ((int)blockIdx.x < p.units) ok = stage_rows(blockIdx.x, 0);
+                for (int u = blockIdx.x; ok && u < p.units; u += gridDim.x, ++n) {
+                    const TcUnit un = tc_unit(p, u, BN);
+                    if (u + (int)gridDim.x < p.units && !(ok = stage_rows(u + gridDim.x, n + 1))) break;
+                    for (int kb = un.kb0; kb < un.kb1; ++kb, ++it) {
+                        const int s = it % STAGES;
+                        const uint32_t ph = (it / STAGES) & 1;
+                        if (!(ok = mbar_wait(&sm.empty[s], ph ^ 1, abort_flag))) break;
+                        mbar_arrive_expect_tx(&sm.full[s], BN * TC_BK);
+                        tma_load_2d(sm.wgt[s], &map_wgt, &sm.full[s], kb * TC_BK, un.c0);
+                    }
+                }
             }
             // gave up: let the copies issued last land before the CTA exits
             if (!ok) {
-                mbar_wait(&sm.w_full, 0, abort_flag);
-                if (n > 0) mbar_wait(&sm.in_full[(n - 1) & 1], ((n - 1) >> 1) & 1, abort_flag);
+                if (LOWER == 1) mbar_wait(&sm.w_full, 0, abort_flag);
+                if (staged > 0) mbar_wait(&sm.in_full[(staged - 1) & 1], ((staged - 1) >> 1) & 1, abort_flag);
             }
         }
         __syncwarp();
@@ -746,14 +774,15 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
             const int b = pix / p.cv_OHW, r = pix - b * p.cv_OHW, oh = r / p.cv_OW, ow = r - oh * p.cv_OW;
             long long lo, hi;
             lw_range(p, un.p0, min(un.p0 + TC_BP, p.N) - 1, &lo, &hi);
-            const int off = (int)((((long long)b * p.lw_H + (long long)oh * p.cv_stride) * p.lw_rowbytes +
-                                   (long long)ow * p.lw_step) - lo);
+            const int ih0 = oh * p.cv_stride - p.cv_pad, iw0 = ow * p.cv_stride - p.cv_pad;   // first tap
+            const int off = (int)((((long long)b * p.lw_H + ih0) * p.lw_rowbytes + (long long)iw0 * p.cv_C) - lo);
             const int src_px = (int)ib * p.lw_stage_bytes + off;        // byte offset of this pixel's first run in stage_in
             if (!warp_wait(&sm.in_full[ib], (ucount >> 1) & 1, lane, abort_flag)) break;
             // Piece V = 8 * kb + c of the lowered row is piece v of run kh; `so` is its byte offset in
             // stage_in.  Branch-free (selects only), so that the eight pieces of a k-block form one
             // block of independent loads and shifts.
             int v = 0, so = src_px, vleft = total_vecs;
+            int kh = 0, kw = 0, vp = 0;                        // LOWER == 2: filter row, tap in it, piece in the pixel
             bool ok = true;
             for (int kb = un.kb0; kb < un.kb1; ++kb, ++it) {
                 const int s = it % STAGES;
@@ -761,24 +790,43 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
                 if (!(ok = warp_wait(&sm.empty[s], ph ^ 1, lane, abort_flag))) break;
                 const uint32_t row = (smem_u32(sm.act[s]) + (uint32_t)t * TC_BK) ^ (uint32_t)((t & 7) << 4);
                 uint32_t o[TC_BK / 16][4];
+                if (LOWER == 1) {
 #pragma unroll
-                for (int c = 0; c < TC_BK / 16; ++c) {
-                    const bool live = c < vleft, last = v == p.lw_vecs - 1;
-                    // an unaligned 16-byte read: five aligned words and four funnel shifts
-                    const int a = live ? so : src_px;
-                    const uint32_t *w = reinterpret_cast<const uint32_t *>(stage_in) + (a >> 2);
-                    const int sh = (a & 3) * 8;
-                    uint32_t x[5];
+                    for (int c = 0; c < TC_BK / 16; ++c) {
+                        const bool live = c < vleft, last = v == p.lw_vecs - 1;
+                        // an unaligned 16-byte read: five aligned words and four funnel shifts
+                        const int a = live ? so : src_px;
+                        const uint32_t *w = reinterpret_cast<const uint32_t *>(stage_in) + (a >> 2);
+                        const int sh = (a & 3) * 8;
+                        uint32_t x[5];
 #pragma unroll
-                    for (int i = 0; i < 5; ++i) x[i] = w[i];
-                    // No masking: the bytes past a run's end (and the pieces past the last run) meet
-                    // weight bytes that are zero -- the pad columns of the weight rows, or depth
-                    // positions past K, which the weight copy fills with zeros -- so whatever image
-                    // bytes land there add nothing to the integer sums.
+                        for (int i = 0; i < 5; ++i) x[i] = w[i];
+                        // No masking: the bytes past a run's end (and the pieces past the last run) meet
+                        // weight bytes that are zero -- the pad columns of the weight rows, or depth
+                        // positions past K, which the weight copy fills with zeros -- so whatever image
+                        // bytes land there add nothing to the integer sums.
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) o[c][i] = __funnelshift_r(x[i], x[i + 1], sh);
-                    so += last ? p.lw_rowbytes - 16 * (p.lw_vecs - 1) : 16;
-                    v = last ? 0 : v + 1;
+                        for (int i = 0; i < 4; ++i) o[c][i] = __funnelshift_r(x[i], x[i + 1], sh);
+                        so += last ? p.lw_rowbytes - 16 * (p.lw_vecs - 1) : 16;
+                        v = last ? 0 : v + 1;
+                    }
+                } else {
+                    // aligned pieces, each inside one pixel: tap (kh, kw) outside the image reads as zero
+#pragma unroll
+                    for (int c = 0; c < TC_BK / 16; ++c) {
+                        const bool last = v == p.lw_vecs - 1;
+                        const bool inside = c < vleft && (unsigned)(ih0 + kh) < (unsigned)p.lw_H &&
+                                            (unsigned)(iw0 + kw) < (unsigned)p.lw_W;
+                        const uint4 d = *reinterpret_cast<const uint4 *>(stage_in + (inside ? so : (int)ib * p.lw_stage_bytes));
+                        o[c][0] = inside ? d.x : 0u; o[c][1] = inside ? d.y : 0u;
+                        o[c][2] = inside ? d.z : 0u; o[c][3] = inside ? d.w : 0u;
+                        const bool px_end = vp == p.lw_cpp - 1;
+                        so += last ? p.lw_rowbytes - 16 * (p.lw_vecs - 1) : 16;
+                        kw = last ? 0 : (px_end ? kw + 1 : kw);
+                        vp = (last || px_end) ? 0 : vp + 1;
+                        kh += last ? 1 : 0;
+                        v = last ? 0 : v + 1;
+                    }
                 }
                 vleft -= TC_BK / 16;
 #pragma unroll
@@ -838,7 +886,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
         if (lane == 0) {
             uint32_t it = 0, tcount = 0;
             bool ok = true;
-            if (LOWER) ok = mbar_wait(&sm.w_full, 0, abort_flag);
+            if (LOWER == 1) ok = mbar_wait(&sm.w_full, 0, abort_flag);
             for (int u = blockIdx.x; ok && u < p.units; u += gridDim.x, ++tcount) {
                 const uint32_t buf = tcount & 1, acc_ph = (tcount >> 1) & 1;
                 const TcUnit un = tc_unit(p, u, BN);
@@ -855,7 +903,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
                     QNN_TRACE(13, it);
                     if (kb == un.kb0) QNN_TRACE(6, tcount);
                     const uint64_t da = umma_smem_desc(smem_u32(sm.act[s]));
-                    const uint64_t db = umma_smem_desc(smem_u32(LOWER ? w_block(kb) : sm.wgt[s]));
+                    const uint64_t db = umma_smem_desc(smem_u32(LOWER == 1 ? w_block(kb) : sm.wgt[s]));
                     // a channel chunk may hold fewer than 128 real bytes: skip the all-zero MMAs
                     int nk = TC_BK / 32;
                     if (p.taps) {
@@ -1161,7 +1209,7 @@ static qnn_status launch_cfg(const CUtensorMap &ma, const CUtensorMap &mw, const
     size_t smem = sizeof(TcSmem<BN, STAGES, OUT_BITS>) + 1024;
     if (LOWER) {
         smem = tc_lower_base_smem<BN, STAGES, OUT_BITS>() + 2 * (size_t)p.lw_stage_bytes +
-               (p.num_kb > STAGES ? (size_t)(p.num_kb - STAGES) * BN * TC_BK : 0);
+               (LOWER == 1 && p.num_kb > STAGES ? (size_t)(p.num_kb - STAGES) * BN * TC_BK : 0);
         if (smem > TC_SMEM_LIMIT) return QNN_ERR_UNSUPPORTED;
     }
     static size_t attr_smem = 0;          // per instantiation: the largest size configured so far
@@ -1393,31 +1441,46 @@ qnn_status gemm_tc_conv_launch(const qnn_conv_desc *cv, const qnn_gemm_desc *g, 
     return tc_launch(g, cv, W, in, thr, out, s);
 }
 
-// Convolution of an 8-bit map whose channel count is not a multiple of 16 (the 3-channel first
-// layer) with the lowering done inside the kernel; weights in the run-per-filter-row layout of
-// qnn_conv_lowered_k.  UNSUPPORTED: padding, a pixel pitch other than C, more than 128 output
-// channels, or weights plus staged image rows that do not fit shared memory -- the caller then
-// lowers explicitly.
-constexpr int LW_BN = 128, LW_STAGES = 4;
+// Convolution of an 8-bit map with contiguous pixels, lowered inside the kernel (see TcParams).
+// Mode 1: channel count not a multiple of 16 (the 3-channel first layer), no padding, at most 128
+// output channels; weights in the run-per-filter-row layout of qnn_conv_lowered_k.  Mode 2: channel
+// count a multiple of 16 but not of 128 (the tensor-map loader would spend a whole k-block on a
+// partly filled channel chunk), any padding smaller than the filter, many tiles.  UNSUPPORTED:
+// everything else, or staged image rows that do not fit shared memory -- the caller then takes
+// another route.
+constexpr int LW_BN = 128, LW_STAGES = 4;          // mode 1
+constexpr int LW2_BN = 256, LW2_STAGES = 3;        // mode 2
 qnn_status gemm_tc_lower_launch(const qnn_conv_desc *cv, const qnn_gemm_desc *g, const void *W, const void *in,
                                 const int32_t *thr, void *out, cudaStream_t s) {
     const int pitch = cv->in_pitch ? cv->in_pitch : round_up(cv->C, 16);
-    if (cv->fmt != QNN_FMT_INT8 || (cv->C % 16) == 0 || pitch != cv->C || cv->pad != 0) return QNN_ERR_UNSUPPORTED;
+    if (cv->fmt != QNN_FMT_INT8 || pitch != cv->C) return QNN_ERR_UNSUPPORTED;
+    const int mode = (cv->C % 16) != 0 ? 1 : 2;
     const int run = cv->KW * cv->C, runp = round_up(run, 16);
     if (g->K != cv->KH * runp) return QNN_ERR_UNSUPPORTED;
     const int OH = qnn_conv_out_h(cv), OW = qnn_conv_out_w(cv);
     if ((long long)g->N * g->K >= (1ll << 40)) return QNN_ERR_UNSUPPORTED;
+    const int bn = mode == 1 ? LW_BN : LW2_BN;
+    const long long tiles = (long long)ceil_div(g->N, TC_BP) * ceil_div(g->M, bn);
+    if (tiles > 0x3fffffff) return QNN_ERR_UNSUPPORTED;
+    if (mode == 1) {
+        // the whole weight matrix stays in shared memory: one channel tile
+        if (cv->pad != 0 || g->M > LW_BN) return QNN_ERR_UNSUPPORTED;
+    } else {
+        const char *force = getenv("QNN_CONV_LOWER");            // "1": skip the heuristic (tests)
+        if (cv->pad >= cv->KH || cv->pad >= cv->KW) return QNN_ERR_UNSUPPORTED;
+        if (!(force && force[0] == '1') && ((cv->C % TC_BK) == 0 || tiles < 2 * sm_count())) return QNN_ERR_UNSUPPORTED;
+    }
 
     TcParams p;
     p.thr = thr; p.out = out; p.M = g->M; p.N = g->N; p.K = g->K;
     p.num_kb = ceil_div(g->K, TC_BK);
     p.ld_out = round_up(g->M, 16);
     p.kb_half = 0; p.share = 0;
-    p.taps = 0; p.cchunks = 1; p.cv_C = cv->C; p.cv_KW = cv->KW; p.cv_pad = 0;
+    p.taps = 0; p.cchunks = 1; p.cv_C = cv->C; p.cv_KW = cv->KW; p.cv_pad = cv->pad;
     p.cv_stride = cv->stride; p.cv_OW = OW; p.cv_OHW = OH * OW;
     p.lw_in = reinterpret_cast<const uint8_t *>(in);
     p.lw_total = (long long)cv->B * cv->H * cv->W * cv->C;
-    p.lw_H = cv->H; p.lw_KH = cv->KH;
+    p.lw_H = cv->H; p.lw_KH = cv->KH; p.lw_W = cv->W; p.lw_cpp = cv->C / 16;
     p.lw_rowbytes = cv->W * cv->C; p.lw_step = cv->stride * cv->C;
     p.lw_run = run; p.lw_vecs = runp / 16;
     // Most image rows a tile of TC_BP consecutive output pixels touches: KH rows for its first
@@ -1430,14 +1493,7 @@ qnn_status gemm_tc_lower_launch(const qnn_conv_desc *cv, const qnn_gemm_desc *g,
     const long long stage = rows * p.lw_rowbytes + 16 + 48;          // rounding of the start, reads past a run
     if (stage > (long long)TC_SMEM_LIMIT) return QNN_ERR_UNSUPPORTED;
     p.lw_stage_bytes = (int)round_up((int)stage, 128);
-    // the whole weight matrix stays in shared memory: one channel tile, a few k-blocks
-    if (g->M > LW_BN) return QNN_ERR_UNSUPPORTED;
-    const size_t w_extra = p.num_kb > LW_STAGES ? (size_t)(p.num_kb - LW_STAGES) * LW_BN * TC_BK : 0;
-    if (tc_lower_base_smem<LW_BN, LW_STAGES, 4>() + 2 * (size_t)p.lw_stage_bytes + w_extra > TC_SMEM_LIMIT)
-        return QNN_ERR_UNSUPPORTED;
-    p.tiles_p = ceil_div(g->N, TC_BP); p.tiles_c = 1;
-    const long long tiles = (long long)p.tiles_p * p.tiles_c;
-    if (tiles > 0x3fffffff) return QNN_ERR_UNSUPPORTED;
+    p.tiles_p = ceil_div(g->N, TC_BP); p.tiles_c = ceil_div(g->M, bn);
     p.units = p.full_units = (int)tiles;
     const double wmax = g->w_enc == QNN_ENC_BIPOLAR ? 1.0
                         : (g->w_enc == QNN_ENC_SIGNED ? double(1 << (g->w_bits - 1)) : double((1 << g->w_bits) - 1));
@@ -1446,11 +1502,13 @@ qnn_status gemm_tc_lower_launch(const qnn_conv_desc *cv, const qnn_gemm_desc *g,
     p.fp_count = (double(g->K) * wmax * amax < double(FP_LIMIT)) ? 1 : 0;
     const uint32_t w_s8 = g->w_enc == QNN_ENC_UNSIGNED ? 0u : 1u;
     const uint32_t a_s8 = g->a_enc == QNN_ENC_UNSIGNED ? 0u : 1u;
-    p.idesc = (2u << 4) | (a_s8 << 7) | (w_s8 << 10) | ((uint32_t)(LW_BN >> 3) << 17) | ((uint32_t)(TC_BP >> 4) << 24);
-    const int mode = !thr ? OUT_RAW : (g->out_fmt == QNN_FMT_INT8 ? OUT_U8 : OUT_PLANES);
+    p.idesc = (2u << 4) | (a_s8 << 7) | (w_s8 << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(TC_BP >> 4) << 24);
+    const int out_mode = !thr ? OUT_RAW : (g->out_fmt == QNN_FMT_INT8 ? OUT_U8 : OUT_PLANES);
     CUtensorMap mw;
-    if (!make_map(&mw, W, g->M, g->K, round_up(g->K, 16), LW_BN)) return QNN_ERR_CUDA;
-    return launch_out<LW_BN, LW_STAGES, 1>(mode, g->out_bits, mw, mw, p, s);
+    if (!make_map(&mw, W, g->M, g->K, round_up(g->K, 16), bn)) return QNN_ERR_CUDA;
+    // shared memory is checked per instantiation (it depends on the number of thresholds)
+    if (mode == 1) return launch_out<LW_BN, LW_STAGES, 1>(out_mode, g->out_bits, mw, mw, p, s);
+    return launch_out<LW2_BN, LW2_STAGES, 2>(out_mode, g->out_bits, mw, mw, p, s);
 }
 
 #ifdef QNN_TC_TRACE

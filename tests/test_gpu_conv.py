@@ -375,3 +375,49 @@ def test_convolution_lowered_inside_the_kernel(qb, monkeypatch, shape):
     assert torch.equal(raw, raw_explicit)
     acc = np.frombuffer(raw.cpu().numpy().tobytes(), dtype=np.int32).reshape(npix, case.OC)
     assert np.array_equal(acc, orc.conv_direct(case.In, case.Wt, case.stride, case.pad).reshape(npix, case.OC))
+
+
+@pytest.mark.parametrize("shape,fits", [
+    # B, H, W, C, OC, KH, KW, stride, pad, w_bits, a_bits; fits: the staged image rows fit shared memory
+    ((2, 27, 27, 96, 256, 5, 5, 1, 2, 1, 2), True),       # conv2 shape: runs of 480 bytes, padding 2
+    ((3, 12, 12, 32, 64, 3, 3, 2, 0, 1, 2), True),        # stride 2, no padding
+    ((2, 23, 17, 16, 48, 5, 3, 3, 2, 2, 2), True),        # stride 3 with padding, rectangular filter and image
+    ((5, 6, 7, 48, 40, 3, 2, 1, 0, 2, 2), True),          # ragged everything
+    ((200, 4, 4, 16, 70, 2, 2, 1, 1, 4, 4), True),        # many small images: a tile spans eight of them
+    ((1, 5, 5, 272, 33, 5, 5, 1, 4, 3, 3), True),         # padding of four around a 5 x 5 map, 17 pieces per pixel
+    ((1, 6, 40, 128, 130, 3, 3, 1, 1, 1, 2), True),       # a full 128-byte channel chunk
+    ((1, 9, 9, 32, 300, 3, 3, 1, 1, 2, 2), True),         # two channel tiles of 256
+    ((4, 9, 9, 128, 130, 3, 3, 2, 1, 1, 2), False),       # 55 image rows of 1152 bytes per tile: another route
+])
+def test_aligned_convolution_lowered_inside_the_kernel(qb, monkeypatch, shape, fits):
+    """8-bit maps with contiguous pixels and C a multiple of 16: the lowering warps copy aligned
+    16-byte pieces (zeros for taps outside the image), weights stream through the ring.  Forced
+    here (the library picks this route for many tiles and C not a multiple of 128); against the
+    direct convolution, the tensor-map loader and the explicit lowering."""
+    monkeypatch.setenv("QNN_CONV_LOWER", "1")
+    case = synth.conv_case(1400 + shape[3] + shape[7], *shape)
+    x, pitch = device_map(qb, case, INT8)
+    assert pitch == case.C
+    Wp = device_weights(qb, case, INT8)
+    npix = case.B * case.OH * case.OW
+    thr = torch.from_numpy(case.thr).cuda()
+    want = orc.qconv(case.In, case.Wt, case.thr, case.stride, case.pad).reshape(npix, case.OC)
+    for out_fmt in (INT8, BITPLANES):
+        d = conv_desc(qb, case, INT8, out_fmt, pitch)
+        n0 = qb.qnn_launch_count()
+        out = qb.qconv(d, Wp, x, thr)
+        if fits:
+            assert qb.qnn_launch_count() - n0 == 1
+        torch.cuda.synchronize()
+        st, dev = qb.qnn_device_status()
+        assert st == 0 and dev == 0
+        assert np.array_equal(decode_out(out.cpu().numpy(), out_fmt, case.out_bits, npix, case.OC, False), want)
+    d = conv_desc(qb, case, INT8, INT8, pitch)
+    raw = qb.qconv(d, Wp, x, None).clone()
+    monkeypatch.delenv("QNN_CONV_LOWER")
+    monkeypatch.setenv("QNN_CONV_IMPLICIT", "1")
+    raw_tma = qb.qconv(d, Wp, x, None).clone()
+    monkeypatch.setenv("QNN_CONV_EXPLICIT", "1")
+    raw_explicit = qb.qconv(d, Wp, x, None)
+    torch.cuda.synchronize()
+    assert torch.equal(raw, raw_explicit) and torch.equal(raw_tma, raw_explicit)
