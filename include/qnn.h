@@ -32,7 +32,8 @@
  *   QNN_TC_NO_SHARE=1          never split a tile's depth between two CTAs
  *   QNN_CONV_EXPLICIT=1        qnn_qconv always goes through the lowered matrix
  *   QNN_CONV_IMPLICIT=1        qnn_qconv lowers inside the GEMM wherever it can
- *   QNN_CONV_LOWER=1           qnn_qconv uses the lowering warps wherever they apply
+ *   QNN_CONV_LOWER=1|0         qnn_qconv uses the aligned lowering warps wherever they
+ *                              apply | never
  *
  * Operand formats
  *   QNN_FMT_BITPLANES  uint32 [bits][rows][kw], kw = ceil(K/32): plane i holds

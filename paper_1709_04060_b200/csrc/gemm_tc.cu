@@ -1445,7 +1445,8 @@ qnn_status gemm_tc_conv_launch(const qnn_conv_desc *cv, const qnn_gemm_desc *g, 
 // Mode 1: channel count not a multiple of 16 (the 3-channel first layer), no padding, at most 128
 // output channels; weights in the run-per-filter-row layout of qnn_conv_lowered_k.  Mode 2: channel
 // count a multiple of 16 but not of 128 (the tensor-map loader would spend a whole k-block on a
-// partly filled channel chunk), any padding smaller than the filter, many tiles.  UNSUPPORTED:
+// partly filled channel chunk), any padding smaller than the filter, at least four rounds of tiles
+// (measured on the 27 x 27 x 96 -> 256 layer: 43 vs 41 us at batch 64, 69 vs 72 at 128, 130 vs 146 at 256).  UNSUPPORTED:
 // everything else, or staged image rows that do not fit shared memory -- the caller then takes
 // another route.
 constexpr int LW_BN = 128, LW_STAGES = 4;          // mode 1
@@ -1466,9 +1467,10 @@ qnn_status gemm_tc_lower_launch(const qnn_conv_desc *cv, const qnn_gemm_desc *g,
         // the whole weight matrix stays in shared memory: one channel tile
         if (cv->pad != 0 || g->M > LW_BN) return QNN_ERR_UNSUPPORTED;
     } else {
-        const char *force = getenv("QNN_CONV_LOWER");            // "1": skip the heuristic (tests)
+        const char *force = getenv("QNN_CONV_LOWER");            // "1": skip the heuristic (tests), "0": never
+        if (force && force[0] == '0') return QNN_ERR_UNSUPPORTED;
         if (cv->pad >= cv->KH || cv->pad >= cv->KW) return QNN_ERR_UNSUPPORTED;
-        if (!(force && force[0] == '1') && ((cv->C % TC_BK) == 0 || tiles < 2 * sm_count())) return QNN_ERR_UNSUPPORTED;
+        if (!(force && force[0] == '1') && ((cv->C % TC_BK) == 0 || tiles < 4 * sm_count())) return QNN_ERR_UNSUPPORTED;
     }
 
     TcParams p;
