@@ -519,7 +519,7 @@ def run_shapes(args):
 # dram__bytes_read.sum + dram__bytes_write.sum of one 4096^3 W1A2 launch of the tensor-core
 # kernel, from the ncu capture summarised in profiles/qgemm_tc_4096_w1a2_w4a4.md (the output
 # codes were still in L2 when the capture ended, so the write counter is small).
-TRAFFIC_BYTES_PER_LAUNCH = 33659648 + 63488
+TRAFFIC_BYTES_PER_LAUNCH = 33657088 + 39936
 
 
 def main():
