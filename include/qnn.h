@@ -28,7 +28,8 @@
  *   QNN_ENC_BIPOLAR   1 bit, bit 1 -> +1, bit 0 -> -1
  *
  * Environment switches (read at call time; for measurements and tests only)
- *   QNN_TC_KERNEL=single|pair  one-CTA (default) or CTA-pair tensor-core kernel
+ *   QNN_TC_KERNEL=single|pair  one-CTA or CTA-pair tensor-core kernel (default: the pair
+ *                              kernel for large problems, the one-CTA kernel otherwise)
  *   QNN_TC_NO_SHARE=1          never split a tile's depth between two CTAs
  *   QNN_CONV_EXPLICIT=1        qnn_qconv always goes through the lowered matrix
  *   QNN_CONV_IMPLICIT=1        qnn_qconv lowers inside the GEMM wherever it can

@@ -174,6 +174,7 @@ def test_partial_last_round_is_shared_by_cta_pairs(qb, monkeypatch, M, N, K, w, 
     depth each; the odd CTA hands its int32 partial sums to the even one through distributed
     shared memory before the threshold epilogue.  Every output is checked, and the same
     problem with sharing switched off must give identical bytes."""
+    monkeypatch.setenv("QNN_TC_KERNEL", "single")     # the larger shapes would otherwise take the CTA-pair kernel
     case = synth.gemm_case(1200 + M, M, N, K, w, a)
     run_case(qb, case, INT8, INT8)
     run_case(qb, case, INT8, BITPLANES)
