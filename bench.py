@@ -385,6 +385,28 @@ def run_extras(args):
     res = {"workload": "extras", "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"]}
 
     only = args.extras_only
+    # ---- large GEMMs (config 5 at N = 8192 and a many-column layer): one-CTA vs CTA-pair kernel
+    large = []
+    for (Mg, Ng, Kg) in ((8192, 8192, 8192), (4096, 18944, 4096), (4096, 18944, 512)) if only in (None, "large") else ():
+        nsets = 2
+        sets = [(torch.randint(-2, 2, (Mg, Kg), dtype=torch.int8, device="cuda"),
+                 torch.randint(0, 4, (Ng, Kg), dtype=torch.uint8, device="cuda")) for _ in range(nsets)]
+        thr_l = torch.sort(torch.randint(-300, 300, (Mg, 3), dtype=torch.int32, device="cuda"), dim=1).values.contiguous()
+        out_l = torch.empty(Ng * Mg, dtype=torch.uint8, device="cuda")
+        dl = qb.gemm_desc(Mg, Ng, Kg, 2, 2, 2, qb.QNN_ENC_SIGNED, qb.QNN_ENC_UNSIGNED, I8, I8)
+        row = {"M": Mg, "N": Ng, "K": Kg}
+        for kern in ("single", "pair", "default"):
+            if kern == "default":
+                os.environ.pop("QNN_TC_KERNEL", None)
+            else:
+                os.environ["QNN_TC_KERNEL"] = kern
+            ms_l = _time_calls(torch, lambda i: qb.check(qb.qnn_qgemm(dl, sets[i % nsets][0], sets[i % nsets][1], thr_l, out_l)),
+                               8, graph=True)
+            row[kern + "_us"] = round(1e3 * ms_l, 1)
+        row["tmacs_default"] = round(Mg * Ng * Kg / (row["default_us"] * 1e-6) / 1e12, 1)
+        large.append(row)
+        del sets, thr_l, out_l
+    res["large_gemm"] = large
     # ---- config 5: M = K = 8192, N in {1, 4, 16}; W2A2 and W4A4
     M = K = 8192
     skinny = []
@@ -532,7 +554,7 @@ def main():
     ap.add_argument("--no-alexnet", action="store_true", help="skip the AlexNet-shaped chain measurement")
     ap.add_argument("--overlap", type=int, default=1,
                     help="1: activation packer on a second stream, overlapping the previous GEMM (default); 0: one stream")
-    ap.add_argument("--extras-only", default=None, choices=["skinny", "conv2", "alexnet"],
+    ap.add_argument("--extras-only", default=None, choices=["large", "skinny", "conv2", "alexnet"],
                     help="extras: run one group only")
     ap.add_argument("--quick", action="store_true",
                     help="extras: a couple of plain calls per case (for profiler captures; AlexNet at batch 32)")

@@ -1290,7 +1290,7 @@ static qnn_status launch_pair_out(int mode, int out_bits, const CUtensorMap &ma,
 
 // Kernel choice.  QNN_TC_KERNEL=single|pair in the environment overrides it (tests, sweeps).
 // The CTA-pair kernel (each SM pulls 32 KB instead of 48 KB per k-block, six stages instead of
-// four) wins on large problems: by 9-18 % at 4096 x 18944 x 512..4096, 8192^3 and
+// four) wins on large problems: by 9-21 % at 4096 x 18944 x 512..4096, 8192^3 and
 // 512 x 75776 x 4096 (eight rounds of SM pairs or more).  Below that the one-CTA kernel stays: its
 // shared last round and programmatic launch count for more (at 4096^3 the pair kernel is 3 % faster
 // back to back with 3 thresholds, slower with 15, and 3 % slower inside the benchmark's
