@@ -323,7 +323,7 @@ def run_b200(args):
         "roofline": {"bound": "tensor", "achieved": achieved_tops, "peak": tensor_peak, "unit": "TOP/s",
                      "frac": achieved_tops / tensor_peak,
                      "traffic": TRAFFIC_BYTES_PER_LAUNCH,
-                     "kernel": "qgemm_tc_kernel (4096^3, int8 operands)",
+                     "kernel": "qgemm_tc2_kernel (CTA-pair tcgen05 kernel, 4096^3, int8 operands)",
                      "peak_source": f"2 x {peaks['source']} bf16 sustained cuBLAS TFLOP/s (nominal int8:bf16 ratio)",
                      "avg_launch_ms": gemm_avg_ms, "algorithmic_ops_per_launch": 2.0 * DIM ** 3},
         "per_pair_tmacs": per_pair,
@@ -538,10 +538,10 @@ def run_shapes(args):
                       "bitplanes_faster": n_bit, "rows": rows}))
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one 4096^3 W1A2 launch of the tensor-core
-# kernel, from the ncu capture summarised in profiles/qgemm_tc_4096_w1a2_w4a4.md (the output
+# dram__bytes_read.sum + dram__bytes_write.sum of one 4096^3 W1A2 launch of the (CTA-pair)
+# tensor-core kernel, from the ncu capture summarised in profiles/qgemm_tc2_4096_w1a2_w4a4.md (the output
 # codes were still in L2 when the capture ended, so the write counter is small).
-TRAFFIC_BYTES_PER_LAUNCH = 33657088 + 39936
+TRAFFIC_BYTES_PER_LAUNCH = 33648384 + 79360
 
 
 def main():

@@ -1047,6 +1047,10 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_const
     tc_fence_before();
     cluster_sync_all();
     tc_fence_after();
+    // set-up done (see the one-CTA kernel): dependents may be placed, and no global memory is
+    // touched before the kernel ahead of this one has completed
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint32_t tmem_base = sm.tmem_base;
     const int num_tiles = p.tiles_p * p.tiles_c;       // tiles of 256 pixels x 256 channels
 
@@ -1258,7 +1262,18 @@ static qnn_status launch_pair_cfg(const CUtensorMap &ma, const CUtensorMap &mw, 
     const int tiles = p.tiles_p * p.tiles_c;
     const int max_pairs = sm_count() / 2;
     const int pairs = tiles < max_pairs ? tiles : max_pairs;
-    kern<<<2 * pairs, TC_THREADS, smem, s>>>(ma, mw, p);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(TC_THREADS);
+    cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    int na = 0;
+    if (2 * pairs >= sm_count() - 1) {     // a grid that fills the GPU: programmatic dependent launch (see launch_cfg)
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    cfg.attrs = attr; cfg.numAttrs = na;
+    if (cudaLaunchKernelEx(&cfg, kern, ma, mw, p) != cudaSuccess) return QNN_ERR_CUDA;
     count_launch();
     return launch_status();
 }
@@ -1290,18 +1305,17 @@ static qnn_status launch_pair_out(int mode, int out_bits, const CUtensorMap &ma,
 
 // Kernel choice.  QNN_TC_KERNEL=single|pair in the environment overrides it (tests, sweeps).
 // The CTA-pair kernel (each SM pulls 32 KB instead of 48 KB per k-block, six stages instead of
-// four) wins on large problems: by 9-21 % at 4096 x 18944 x 512..4096, 8192^3 and
-// 512 x 75776 x 4096 (eight rounds of SM pairs or more).  Below that the one-CTA kernel stays: its
-// shared last round and programmatic launch count for more (at 4096^3 the pair kernel is 3 % faster
-// back to back with 3 thresholds, slower with 15, and 3 % slower inside the benchmark's
-// packer + GEMM sequence).
+// four) is the faster one wherever its 256 x 256 tiles fill the SM pairs for a round and a half or
+// more and waste little of N: by 6 % on the 4096^3 sweep inside the packer + GEMM sequence, by
+// 12-22 % at 4096 x 18944 x 512..4096 and 8192^3 (tensor pipe 88 % busy).  Smaller problems keep the
+// one-CTA kernel, whose tiles of the last round are shared by CTA pairs that split the depth.
 static bool choose_pair_kernel(const qnn_gemm_desc *d, int sms) {
     const char *force = getenv("QNN_TC_KERNEL");
     if (force && force[0] == 's') return false;
     if (force && force[0] == 'p') return true;
     const int pairs = sms / 2;
     const long long tiles2 = (long long)ceil_div(d->N, 256) * ceil_div(d->M, T2_BN);
-    return d->M >= T2_BN && d->N >= 2048 && tiles2 >= 8ll * pairs;
+    return d->M >= T2_BN && d->N >= 2048 && 2 * tiles2 >= 3ll * pairs;
 }
 
 // Tile plan of the one-CTA kernel: channel tile, grid, and whether the tiles of the last
