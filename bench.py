@@ -369,6 +369,79 @@ def _time_calls(torch, fn, iters, warmup=3, graph=False):
     return e0.elapsed_time(e1) / iters
 
 
+def measure_peaks(torch, qb, mma_configs=((1, 256),), mmas=4096, popc_iters=4096, reps=5):
+    """Issue-bound peaks of the two GEMM paths, timed with CUDA events (best of `reps`):
+    tcgen05 kind::i8 MMAs on shared-memory-resident tiles (pair: cta_group::2) and XOR+POPC
+    chains.  Returns {"mma_i8": {"pair<p>_n<n>": TOP/s, ...}, "popc_g_per_s": ..}."""
+    out = {"mma_i8": {}}
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for (pair, n) in mma_configs:
+        best = None
+        for r in range(reps + 1):
+            e0.record()
+            st, ops = qb.qnn_peak_mma_i8(pair, n, mmas)
+            e1.record()
+            qb.check(st)
+            torch.cuda.synchronize()
+            if r > 0:
+                ms = e0.elapsed_time(e1)
+                best = ms if best is None else min(best, ms)
+        out["mma_i8"][f"pair{pair}_n{n}"] = round(ops / (best * 1e-3) / 1e12, 1)
+    sink = torch.empty(qb.qnn_peak_popc_sink_bytes(), dtype=torch.uint8, device="cuda")
+    best = None
+    for r in range(reps + 1):
+        e0.record()
+        st, popcs = qb.qnn_peak_popc(popc_iters, sink)
+        e1.record()
+        qb.check(st)
+        torch.cuda.synchronize()
+        if r > 0:
+            ms = e0.elapsed_time(e1)
+            best = ms if best is None else min(best, ms)
+    out["popc_g_per_s"] = round(popcs / (best * 1e-3) / 1e9, 1)
+    out["binary_tmac_per_s"] = round(32 * popcs / (best * 1e-3) / 1e12, 2)
+    st, dev = qb.qnn_device_status()
+    assert st == 0 and dev == 0
+    return out
+
+
+def run_peaks(args):
+    """Roofline denominators measured on this GPU: the int8 tensor-pipe issue rate for a range of
+    MMA widths (one CTA per SM, and CTA pairs) and the POPC issue rate, with the SM clock sampled
+    meanwhile.  Prints one JSON line."""
+    import torch
+    import __graft_entry__ as ge
+    ge.build()
+    from paper_1709_04060_b200 import binding as qb
+    torch.cuda.set_device(0)
+    sampler = ClockSampler(0)
+    sampler.start()
+    time.sleep(0.15)
+    t0 = time.time()
+    cfgs = [(0, n) for n in (16, 32, 64, 128, 256)] + [(1, n) for n in (32, 64, 128, 256)]
+    res = measure_peaks(torch, qb, cfgs, mmas=16384, popc_iters=16384, reps=8)
+    # a seconds-long run of the widest pair MMA: the sustained figure under the power cap
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    total = 0.0
+    for _ in range(60):
+        st, ops = qb.qnn_peak_mma_i8(1, 256, 65536)
+        qb.check(st)
+        total += ops
+    e1.record()
+    torch.cuda.synchronize()
+    res["mma_i8_sustained_pair1_n256"] = round(total / (e0.elapsed_time(e1) * 1e-3) / 1e12, 1)
+    res["sustained_seconds"] = round(e0.elapsed_time(e1) * 1e-3, 2)
+    clocks = sampler.stop(t0, time.time())
+    peaks = load_peaks()
+    res.update({"workload": "peaks", "clocks": clocks,
+                "nominal": {"int8_dense_tops": 4500.0, "popc_per_clk_per_sm": 16,
+                            "popc_g_per_s_at_max_clock": 16 * 148 * 1.965},
+                "measured_bf16_tflops": {"burst": peaks["bf16_burst"], "sustained": peaks["bf16_sustained"],
+                                         "source": peaks["source"]}})
+    print(json.dumps(res))
+
+
 def run_extras(args):
     """The other paper-shaped workloads on one GPU (not the headline line): the large/skinny
     fully connected sweep (HBM roofline, weight buffers rotated so that every call streams
@@ -558,7 +631,7 @@ def main():
                     help="extras: run one group only")
     ap.add_argument("--quick", action="store_true",
                     help="extras: a couple of plain calls per case (for profiler captures; AlexNet at batch 32)")
-    ap.add_argument("--workload", default="sweep", choices=["sweep", "extras", "shapes"],
+    ap.add_argument("--workload", default="sweep", choices=["sweep", "extras", "shapes", "peaks"],
                     help="sweep: the headline line; extras: the other paper-shaped workloads (one GPU); "
                          "shapes: the 2^6..2^12 size sweep of both operand formats")
     ap.add_argument("--pairs", default=None,
@@ -566,10 +639,10 @@ def main():
     args = ap.parse_args()
     if args.pairs:
         PAIRS[:] = [tuple(int(v) for v in p.split("x")) for p in args.pairs.split(",")]
-    if args.workload in ("extras", "shapes"):
+    if args.workload in ("extras", "shapes", "peaks"):
         global QUICK
         QUICK = args.quick
-        (run_extras if args.workload == "extras" else run_shapes)(args)
+        {"extras": run_extras, "shapes": run_shapes, "peaks": run_peaks}[args.workload](args)
         return
     if args.impl == "reference":
         if args.steps is None:

@@ -44,8 +44,9 @@
  *                      activations, its channel-interleaved layout (Section 3.2).
  *   QNN_FMT_INT8       one byte per element [rows][ld], ld = K rounded up to a
  *                      multiple of 16, pad bytes zero: int8 for SIGNED/BIPOLAR,
- *                      uint8 for UNSIGNED (Section 3: "casting all operands to
- *                      8-bit integers"); the tensor-core path consumes this.
+ *                      uint8 for UNSIGNED (the 8-bit formulation of Section 3:
+ *                      few-bit values held in 8-bit containers); the tensor-core
+ *                      path consumes this.
  */
 #ifndef QNN_H_
 #define QNN_H_
@@ -255,6 +256,26 @@ typedef struct {
  * pointers; nothing is launched.  Errors: INVALID_ARG. */
 qnn_status qnn_streamline(const qnn_channel_params *ch, int channels, const double *qthr, int n_thr,
                           long long acc_lo, long long acc_hi, int32_t *thr_out, uint8_t *negate_out);
+
+/* ---- roofline denominators (Section 4.1.1 reports against the machine's peak) -- */
+
+/* Launches the tensor-pipe issue-rate microbenchmark on `stream`: every SM (pair == 0; one
+ * CTA each) or every pair of SMs (pair != 0; tcgen05 cta_group::2) issues mmas_per_cta
+ * back-to-back tcgen05.mma kind::i8 instructions of 128 (256 for a pair) x n x 32 on operand
+ * tiles resident in shared memory: no loads, no epilogue.  n: a multiple of 16 (32 for a
+ * pair) in [16, 256].  *ops (host) receives the integer operations (2 per multiply-
+ * accumulate) the launch performs; the caller times the launch with events.  The peak of
+ * the dense int8 tensor path is ops / time.  Errors: INVALID_ARG, CUDA. */
+qnn_status qnn_peak_mma_i8(int pair, int n, int mmas_per_cta, double *ops, void *stream);
+
+/* Launches the POPC issue-rate microbenchmark (chains of XOR + POPC in registers, the inner
+ * operation of Algorithm 1): *popcs (host) receives the number of 32-bit population counts
+ * the launch executes; 32 x popcs / time is the peak of the bit-serial path in binary
+ * multiply-accumulates per second.  sink: device scratch of at least
+ * qnn_peak_popc_sink_bytes() bytes, 16-byte aligned (each thread stores one word there).
+ * Errors: INVALID_ARG, WORKSPACE, ALIGNMENT, CUDA. */
+qnn_status qnn_peak_popc(int iters, void *sink, size_t sink_bytes, double *popcs, void *stream);
+size_t qnn_peak_popc_sink_bytes(void);
 
 /* ---- utilities ------------------------------------------------------------ */
 

@@ -36,7 +36,7 @@ EXPORTS = (
     "qnn_gemm_out_bytes", "qnn_qgemm", "qnn_conv_out_h", "qnn_conv_out_w",
     "qnn_conv_lowered_k", "qnn_conv_lowered_bytes", "qnn_conv_workspace_bytes",
     "qnn_conv_out_bytes", "qnn_im2col", "qnn_qconv", "qnn_qconv_static", "qnn_maxpool",
-    "qnn_streamline", "qnn_validate_thresholds", "qnn_device_status", "qnn_launch_count",
+    "qnn_streamline", "qnn_peak_mma_i8", "qnn_peak_popc", "qnn_peak_popc_sink_bytes", "qnn_validate_thresholds", "qnn_device_status", "qnn_launch_count",
     "qnn_status_string", "qnn_version",
 )
 
@@ -99,6 +99,12 @@ _lib.qnn_maxpool.argtypes = [_P(qnn_pool_desc), _vp, _vp, _vp]
 _lib.qnn_streamline.restype = _ci
 _lib.qnn_streamline.argtypes = [_P(qnn_channel_params), _ci, _P(ctypes.c_double), _ci, ctypes.c_longlong,
                                 ctypes.c_longlong, _P(ctypes.c_int32), _P(ctypes.c_uint8)]
+_lib.qnn_peak_mma_i8.restype = _ci
+_lib.qnn_peak_mma_i8.argtypes = [_ci, _ci, _ci, _P(ctypes.c_double), _vp]
+_lib.qnn_peak_popc.restype = _ci
+_lib.qnn_peak_popc.argtypes = [_ci, _vp, _sz, _P(ctypes.c_double), _vp]
+_lib.qnn_peak_popc_sink_bytes.restype = _sz
+_lib.qnn_peak_popc_sink_bytes.argtypes = []
 _lib.qnn_validate_thresholds.restype = _ci
 _lib.qnn_validate_thresholds.argtypes = [_vp, _ci, _ci, _P(_ci), _vp]
 _lib.qnn_device_status.restype = _ci
@@ -237,6 +243,25 @@ def qnn_streamline(channels, qthr, acc_lo: int, acc_hi: int):
     st = _lib.qnn_streamline(arr, len(channels), q, n, int(acc_lo), int(acc_hi), out, neg)
     thr = [[out[c * n + i] for i in range(n)] for c in range(len(channels))]
     return st, thr, [int(v) for v in neg]
+
+
+def qnn_peak_mma_i8(pair: int, n: int, mmas_per_cta: int, stream=None):
+    """Launches the tensor-pipe issue-rate microbenchmark; returns (status, integer ops of the launch)."""
+    ops = ctypes.c_double(0.0)
+    st = _lib.qnn_peak_mma_i8(int(pair), int(n), int(mmas_per_cta), ctypes.byref(ops), _stream(stream))
+    return st, ops.value
+
+
+def qnn_peak_popc_sink_bytes() -> int:
+    return int(_lib.qnn_peak_popc_sink_bytes())
+
+
+def qnn_peak_popc(iters: int, sink, stream=None):
+    """Launches the POPC issue-rate microbenchmark; returns (status, population counts of the launch)."""
+    n = ctypes.c_double(0.0)
+    st = _lib.qnn_peak_popc(int(iters), _ptr(sink), sink.numel() * sink.element_size(), ctypes.byref(n),
+                            _stream(stream))
+    return st, n.value
 
 
 def qnn_validate_thresholds(thr, M: int, n_thr: int, stream=None):

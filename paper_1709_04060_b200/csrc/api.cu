@@ -6,7 +6,7 @@
 
 namespace qnn {
 
-unsigned long long g_launches = 0;
+std::atomic<unsigned long long> g_launches{0};
 
 int sm_count() {
     static int cached[64] = {0};
@@ -62,6 +62,10 @@ static qnn_status check_conv_desc(const qnn_conv_desc *d) {
     if (!valid_fmt(d->fmt)) return QNN_ERR_INVALID_ARG;
     if (d->a_bits < 1 || d->a_bits > 8) return QNN_ERR_INVALID_ARG;
     if (d->H + 2 * d->pad < d->KH || d->W + 2 * d->pad < d->KW) return QNN_ERR_INVALID_ARG;
+    // the lowered GEMM's column count B*OH*OW and the map's pixel count are ints
+    const long long oh = (d->H + 2 * d->pad - d->KH) / d->stride + 1, ow = (d->W + 2 * d->pad - d->KW) / d->stride + 1;
+    if ((long long)d->B * oh * ow > 0x7fffffffll || (long long)d->B * d->H * d->W > 0x7fffffffll)
+        return QNN_ERR_UNSUPPORTED;
     if (d->fmt == QNN_FMT_INT8 && d->in_pitch != 0 && d->in_pitch < d->C) return QNN_ERR_INVALID_ARG;
     if (d->a_enc == QNN_ENC_BIPOLAR && d->pad > 0) return QNN_ERR_UNSUPPORTED;
     // per-pixel pad bits would read as -1 for a bipolar operand
@@ -103,7 +107,7 @@ const char *qnn_status_string(qnn_status s) {
     return "unknown status";
 }
 
-unsigned long long qnn_launch_count(void) { return g_launches; }
+unsigned long long qnn_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 size_t qnn_packed_ld(int K, int fmt) {
     if (K <= 0) return 0;

@@ -5,14 +5,26 @@
 #include <stdint.h>
 #include <stddef.h>
 
+#include <atomic>
+
 #include "qnn.h"
 
 namespace qnn {
 
 // Host counter of kernels launched by this library (reported by benchmarks).
-extern unsigned long long g_launches;
+extern std::atomic<unsigned long long> g_launches;
 
-inline void count_launch(int n = 1) { g_launches += (unsigned long long)n; }
+inline void count_launch(int n = 1) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+
+// Per-device host caches are arrays of this size; a device index beyond it is an error.
+constexpr int QNN_MAX_DEVICES = 64;
+
+// Index of the current device, or -1 (CUDA error, or an index the caches cannot hold).
+inline int current_device() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= QNN_MAX_DEVICES) return -1;
+    return dev;
+}
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 

@@ -1,7 +1,7 @@
 // Tensor-core few-bit GEMM fused with the threshold activation.
 //
-// The few-bit operands sit in 8-bit containers (Section 3 of the paper: "casting
-// all operands to 8-bit integers"); on B200 the fifth-generation tensor cores
+// The few-bit operands sit in 8-bit containers (the 8-bit formulation that Section 3
+// of the paper starts from); on B200 the fifth-generation tensor cores
 // multiply them exactly (tcgen05.mma kind::i8, int32 accumulators in tensor
 // memory), which reproduces the integer product that the bit-serial sum of
 // Section 3.1 equals.  The epilogue applies T(x, t) of Section 2.1.1 to the
@@ -44,6 +44,7 @@
 #include <stdlib.h>
 
 #include "common.cuh"
+#include "tc_ptx.cuh"
 
 namespace qnn {
 
@@ -68,132 +69,13 @@ __device__ int g_trace_cta;
 
 constexpr int TC_BP = 128;          // activation rows (pixels) per tile = tensor-memory lanes
 constexpr int TC_BK = 128;          // depth bytes per stage = one 128B swizzle row
-constexpr long long TC_WAIT_CYCLES = 2000000000ll;   // ~1 s
 
-// ---------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void *p) {
-    return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
-                 : "memory");
-}
-// One try: the thread is suspended until the phase completes or the time hint runs out (it
-// issues nothing meanwhile, so waiting roles leave the issue slots to the working ones).
-constexpr uint32_t MBAR_SUSPEND_NS = 20000;
-__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.b32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(MBAR_SUSPEND_NS) : "memory");
-    return ok != 0;
-}
-// Bounded wait.  Returns false if the limit ran out or another role gave up.
+// Waits of this file report to the status word defined here.
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (;;) {
-#pragma unroll 1
-        for (int i = 0; i < 64; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (clock64() - t0 > TC_WAIT_CYCLES) {
-            *abort_flag = 1;
-            atomicExch(&g_dev_status, (int)QNN_ERR_DEVICE_TIMEOUT);
-            return false;
-        }
-    }
+    return mbar_wait(bar, parity, abort_flag, &g_dev_status);
 }
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-// Bounded wait that also acquires what another CTA of the cluster released on the barrier.
 __device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
-    const long long t0 = clock64();
-    for (;;) {
-        uint32_t ok;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
-            "selp.b32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(MBAR_SUSPEND_NS) : "memory");
-        if (ok) return true;
-        if (*abort_flag) return false;
-        if (clock64() - t0 > TC_WAIT_CYCLES) {
-            *abort_flag = 1;
-            atomicExch(&g_dev_status, (int)QNN_ERR_DEVICE_TIMEOUT);
-            return false;
-        }
-    }
-}
-__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, uint64_t *bar, int x, int y) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y) : "memory");
-}
-// im2col-mode load (Section 3.2's lowering done by the copy engine): 128 consecutive output
-// pixels starting at base pixel (w, h, n) of the padded map, filter tap offset (woff, hoff),
-// channels [c, c + 128); pixels outside the image and channels past C read as zero.
-__device__ __forceinline__ void tma_load_im2col(void *dst, const CUtensorMap *map, uint64_t *bar, int c, int w,
-                                                int h, int n, uint16_t woff, uint16_t hoff) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes "
-        "[%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
-        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c), "r"(w), "r"(h), "r"(n), "h"(woff), "h"(hoff)
-        : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t ncols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)),
-                 "r"(ncols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
-__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                        uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint64_t *bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-                 : "memory");
-}
-// K-major operand tile, rows at a 128-byte pitch, 128B swizzle (what TMA writes
-// with CU_TENSOR_MAP_SWIZZLE_128B): 8-row groups are 1024 bytes apart.
-__device__ __forceinline__ uint64_t umma_smem_desc(uint32_t saddr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);          // start address
-    d |= (uint64_t)1 << 16;                            // leading byte offset (unused for swizzled K-major)
-    d |= (uint64_t)(1024 >> 4) << 32;                  // stride byte offset: 8 rows x 128 B
-    d |= (uint64_t)1 << 46;                            // descriptor version of this architecture
-    d |= (uint64_t)2 << 61;                            // 128-byte swizzle
-    return d;
+    return mbar_wait_cluster(bar, parity, abort_flag, &g_dev_status);
 }
 
 struct TcParams {
@@ -989,34 +871,6 @@ struct Tc2Smem {
     int abort_flag;
 };
 
-__device__ __forceinline__ void tma_load_2d_pair(void *dst, const CUtensorMap *map, uint32_t bar_cluster_addr,
-                                                 int x, int y) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
-        "[%0], [%1, {%3, %4}], [%2];"
-        ::"r"(smem_u32(dst)), "l"(map), "r"(bar_cluster_addr), "r"(x), "r"(y) : "memory");
-}
-__device__ __forceinline__ void tmem_alloc_pair(uint32_t *dst_smem, uint32_t ncols) {
-    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)),
-                 "r"(ncols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
-    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
-__device__ __forceinline__ void umma_i8_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                             uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// Arrive on the barrier at cluster address `bar` once all MMAs issued so far are done.
-__device__ __forceinline__ void umma_commit_pair(uint32_t bar_cluster_addr) {
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];"
-                 ::"r"(bar_cluster_addr) : "memory");
-}
-
 template <int OUT_MODE, int OUT_BITS>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_constant__ CUtensorMap map_wgt,
@@ -1216,11 +1070,14 @@ static qnn_status launch_cfg(const CUtensorMap &ma, const CUtensorMap &mw, const
                (LOWER == 1 && p.num_kb > STAGES ? (size_t)(p.num_kb - STAGES) * BN * TC_BK : 0);
         if (smem > TC_SMEM_LIMIT) return QNN_ERR_UNSUPPORTED;
     }
-    static size_t attr_smem = 0;          // per instantiation: the largest size configured so far
-    if (smem > attr_smem) {
+    // per instantiation and device: the largest size configured so far
+    static size_t attr_smem[QNN_MAX_DEVICES] = {0};
+    const int dev = current_device();
+    if (dev < 0) return QNN_ERR_CUDA;
+    if (smem > attr_smem[dev]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return QNN_ERR_CUDA;
-        attr_smem = smem;
+        attr_smem[dev] = smem;
     }
     const int grid = p.units < sm_count() ? p.units : sm_count();
     cudaLaunchConfig_t cfg = {};
@@ -1253,11 +1110,13 @@ template <int OUT_MODE, int OUT_BITS>
 static qnn_status launch_pair_cfg(const CUtensorMap &ma, const CUtensorMap &mw, const TcParams &p, cudaStream_t s) {
     auto kern = qgemm_tc2_kernel<OUT_MODE, OUT_BITS>;
     const size_t smem = sizeof(Tc2Smem<OUT_BITS>) + 1024;
-    static bool attr_done = false;
-    if (!attr_done) {
+    static bool attr_done[QNN_MAX_DEVICES] = {false};       // per instantiation and device
+    const int dev = current_device();
+    if (dev < 0) return QNN_ERR_CUDA;
+    if (!attr_done[dev]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return QNN_ERR_CUDA;
-        attr_done = true;
+        attr_done[dev] = true;
     }
     const int tiles = p.tiles_p * p.tiles_c;
     const int max_pairs = sm_count() / 2;
@@ -1488,6 +1347,10 @@ qnn_status gemm_tc_lower_launch(const qnn_conv_desc *cv, const qnn_gemm_desc *g,
     if (mode == 1) {
         // the whole weight matrix stays in shared memory: one channel tile
         if (cv->pad != 0 || g->M > LW_BN) return QNN_ERR_UNSUPPORTED;
+        // The unaligned runs are not masked: image bytes, not zeros, sit opposite the pad columns
+        // of the weight rows, which therefore have to be zero bytes.  A bipolar weight has no zero
+        // (the packer writes -1 for a logical 0), so such layers take another route.
+        if (g->w_enc == QNN_ENC_BIPOLAR && runp != run) return QNN_ERR_UNSUPPORTED;
     } else {
         const char *force = getenv("QNN_CONV_LOWER");            // "1": skip the heuristic (tests), "0": never
         if (force && force[0] == '0') return QNN_ERR_UNSUPPORTED;
@@ -1543,6 +1406,18 @@ extern "C" int qnn_debug_trace_cta(int cta) {
     return (int)cudaMemcpyToSymbol(g_trace_cta, &cta, sizeof(int));
 }
 #endif
+
+int *device_status_word() {
+    static int *cached[QNN_MAX_DEVICES] = {nullptr};
+    const int dev = current_device();
+    if (dev < 0) return nullptr;
+    if (!cached[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_dev_status) != cudaSuccess) return nullptr;
+        cached[dev] = reinterpret_cast<int *>(p);
+    }
+    return cached[dev];
+}
 
 qnn_status device_status_read(int *status) {
     int v = 0;

@@ -11,17 +11,17 @@
 
 namespace qnn {
 
-struct FastDiv {          // exact n / d for n, d < 65536
+struct FastDiv {          // n / d: by multiplication (exact for n, d < 65536), else magic == 0 and a plain division
     uint32_t d, magic;
 };
-static FastDiv make_fastdiv(int d) {
+static FastDiv make_fastdiv(int d, long long max_n = 0) {
     FastDiv f;
     f.d = (uint32_t)d;
-    f.magic = (uint32_t)(((1ull << 32) + (uint64_t)d - 1) / (uint64_t)d);
+    f.magic = (d >= 65536 || max_n >= 65536) ? 0u : (uint32_t)(((1ull << 32) + (uint64_t)d - 1) / (uint64_t)d);
     return f;
 }
 __device__ __forceinline__ uint32_t fdiv(uint32_t n, FastDiv f) {
-    return f.d == 1 ? n : __umulhi(n, f.magic);
+    return f.d == 1 ? n : (f.magic ? __umulhi(n, f.magic) : n / f.d);
 }
 
 struct LowerParams {
@@ -184,8 +184,7 @@ qnn_status im2col_launch(const qnn_conv_desc *d, const void *in, void *lowered, 
     p.OH = qnn_conv_out_h(d); p.OW = qnn_conv_out_w(d);
     p.KH = d->KH; p.KW = d->KW; p.stride = d->stride; p.pad = d->pad;
     p.npix = (long long)d->B * p.OH * p.OW;
-    if (p.OH * p.OW >= 65536 || p.OW >= 65536) return QNN_ERR_UNSUPPORTED;
-    p.owd = make_fastdiv(p.OW);
+    p.owd = make_fastdiv(p.OW, (long long)p.OH * p.OW);      // large maps: plain division
     const int threads = 256;
     const long long max_blocks = (long long)sm_count() * 16;
 

@@ -377,6 +377,43 @@ def test_convolution_lowered_inside_the_kernel(qb, monkeypatch, shape):
     assert np.array_equal(acc, orc.conv_direct(case.In, case.Wt, case.stride, case.pad).reshape(npix, case.OC))
 
 
+@pytest.mark.parametrize("shape", [
+    # B, H, W, C, OC, KH, KW, stride, pad, w_bits, a_bits
+    (2, 20, 21, 3, 40, 5, 5, 2, 0, 1, 2),         # runs of 15 bytes: one pad column per filter row
+    (3, 9, 9, 5, 17, 3, 3, 1, 0, 1, 2),           # runs of 15 bytes
+    (2, 11, 10, 20, 64, 3, 3, 1, 0, 1, 4),        # runs of 60 bytes
+    (1, 12, 12, 16, 32, 3, 3, 1, 0, 1, 2),        # C a multiple of 16: no pad columns at all
+])
+def test_bipolar_weights_with_unaligned_runs(qb, monkeypatch, shape):
+    """Bipolar weights have no zero: the pad columns that close each filter row's run hold -1 after
+    packing.  The unmasked in-kernel lowering (which leaves image bytes opposite those columns)
+    must therefore not be chosen for such a layer; whatever route the library takes, the codes and
+    accumulators equal the direct convolution and the explicit route."""
+    case = synth.conv_case(1500 + shape[3] + shape[5], *shape)
+    assert case.w_enc == synth.BIPOLAR
+    x, pitch = device_map(qb, case, INT8, in_pitch=case.C)
+    Wp = device_weights(qb, case, INT8)
+    npix = case.B * case.OH * case.OW
+    thr = torch.from_numpy(case.thr).cuda()
+    want = orc.qconv(case.In, case.Wt, case.thr, case.stride, case.pad).reshape(npix, case.OC)
+    want_acc = orc.conv_direct(case.In, case.Wt, case.stride, case.pad).reshape(npix, case.OC)
+    for out_fmt in (INT8, BITPLANES):
+        d = conv_desc(qb, case, INT8, out_fmt, pitch)
+        out = qb.qconv(d, Wp, x, thr)
+        torch.cuda.synchronize()
+        assert np.array_equal(decode_out(out.cpu().numpy(), out_fmt, case.out_bits, npix, case.OC, False), want)
+    d = conv_desc(qb, case, INT8, INT8, pitch)
+    raw = qb.qconv(d, Wp, x, None).clone()
+    acc = np.frombuffer(raw.cpu().numpy().tobytes(), dtype=np.int32).reshape(npix, case.OC)
+    assert np.array_equal(acc, want_acc)
+    monkeypatch.setenv("QNN_CONV_EXPLICIT", "1")
+    raw_explicit = qb.qconv(d, Wp, x, None)
+    torch.cuda.synchronize()
+    assert torch.equal(raw, raw_explicit)
+    st, dev = qb.qnn_device_status()
+    assert st == 0 and dev == 0
+
+
 @pytest.mark.parametrize("shape,fits", [
     # B, H, W, C, OC, KH, KW, stride, pad, w_bits, a_bits; fits: the staged image rows fit shared memory
     ((2, 27, 27, 96, 256, 5, 5, 1, 2, 1, 2), True),       # conv2 shape: runs of 480 bytes, padding 2

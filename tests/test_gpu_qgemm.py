@@ -205,20 +205,29 @@ def test_integer_count_path_for_large_accumulators(qb, force_tc_kernel, which):
     run_case(qb, small, BITPLANES, INT8)
 
 
-@pytest.mark.parametrize("w,a", [(1, 2), (4, 4)])
+def _sample_indices(rng, M, N, count, edges):
+    rows = np.concatenate([rng.integers(0, M, count), [e % M for e in edges]])
+    cols = np.concatenate([rng.integers(0, N, count), [e % N for e in reversed(edges)]])
+    return rows, cols
+
+
+@pytest.mark.parametrize("w,a", list(itertools.product((1, 2, 3, 4), repeat=2)))
 def test_full_size_4096_sampled(qb, w, a):
-    """The benchmark's problem size and launch configuration (M=N=K=4096), checked on
-    sampled outputs the oracle computes one by one, plus whole rows/columns."""
+    """Every problem of the benchmark's sweep in the benchmark's own launch configuration
+    (M = N = K = 4096, 8-bit containers in and out, the library's kernel choice, 2^a - 1
+    thresholds): sampled accumulators and codes against oracle dot products, plus one whole
+    weight row and one whole column.  A bit-plane output of the same problem is decoded and
+    compared with the byte output element by element."""
     case = synth.gemm_case(2000 + 10 * w + a, 4096, 4096, 4096, w, a)
     Wd = qb.to_device_logical(case.W, case.w_enc)
     Ad = qb.to_device_logical(case.At, case.a_enc)
     Wp, Ap = qb.pack(Wd, w, case.w_enc, INT8), qb.pack(Ad, a, case.a_enc, INT8)
     d = qb.gemm_desc(4096, 4096, 4096, w, a, a, case.w_enc, case.a_enc, INT8, INT8)
-    codes = qb.qgemm(d, Wp, Ap, torch.from_numpy(case.thr).cuda()).cpu().numpy().reshape(4096, 4096)
+    thr = torch.from_numpy(case.thr).cuda()
+    codes = qb.qgemm(d, Wp, Ap, thr).cpu().numpy().reshape(4096, 4096)
     raw = qb.qgemm(d, Wp, Ap, None).cpu().numpy()
     rng = np.random.default_rng(7)
-    rows = np.concatenate([rng.integers(0, 4096, 3000), [0, 4095, 127, 128, 255, 256, 4095]])
-    cols = np.concatenate([rng.integers(0, 4096, 3000), [0, 4095, 255, 256, 4095, 0, 0]])
+    rows, cols = _sample_indices(rng, 4096, 4096, 3000, [0, 4095, 127, 128, 255, 256, 4095])
     acc = orc.dot_at(case.W, case.At, rows, cols)
     assert np.array_equal(raw[cols, rows].astype(np.int64), acc)
     want = (acc[:, None] >= case.thr[rows]).sum(axis=1)
@@ -228,6 +237,31 @@ def test_full_size_4096_sampled(qb, w, a):
     assert np.array_equal(codes[:, 777].astype(np.int64), full_row)
     full_col = orc.qgemm(case.W, case.At[1234:1235], case.thr)[:, 0]
     assert np.array_equal(codes[1234, :].astype(np.int64), full_col)
+    # the raw accumulators decide every code: all 16.8 M codes against the counting rule
+    # applied on the host to the device's own accumulators (whose samples the oracle confirmed)
+    recount = np.zeros(raw.shape, dtype=np.uint8)
+    for q in range(case.thr.shape[1]):
+        recount += raw >= case.thr[None, :, q]
+    assert np.array_equal(codes, recount)
+    dp = qb.gemm_desc(4096, 4096, 4096, w, a, a, case.w_enc, case.a_enc, INT8, BITPLANES)
+    planes = qb.qgemm(dp, Wp, Ap, thr).cpu().numpy()
+    assert np.array_equal(decode_out(planes, BITPLANES, a, 4096, 4096, False), codes.astype(np.int64))
+    st, dev = qb.qnn_device_status()
+    assert st == 0 and dev == 0
+
+
+@pytest.mark.parametrize("out_bits", [1, 2, 3, 4])
+def test_pair_kernel_many_rounds_every_threshold_count(qb, force_tc_kernel, out_bits):
+    """The CTA-pair kernel over several rounds of its persistent loop (2 x 157 = 314 tiles of
+    256 x 256 on 74 SM pairs: the tensor-memory and threshold double buffers wrap twice, the
+    last round is partial), for 1, 3, 7 and 15 thresholds and both output layouts: every
+    output against the oracle."""
+    force_tc_kernel("pair")
+    M, N, K = 512, 40000, 256
+    case = synth.gemm_case(1700 + out_bits, M, N, K, 2, out_bits, out_bits=out_bits)
+    run_case(qb, case, INT8, INT8, path=2)
+    run_case(qb, case, INT8, BITPLANES, path=2)
+    run_case(qb, case, INT8, INT8, raw=True, path=2)
 
 
 @pytest.mark.parametrize("fmt", [BITPLANES, INT8])

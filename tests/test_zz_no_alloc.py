@@ -6,7 +6,8 @@ tensors, or a latency-bound loop where cudaMalloc is banned because it may stall
 device.  For them the lowered matrix sits in a fixed 16 MiB array inside the library.
 This file checks, through the C ABI, that the entry point gives exactly what qnn_qconv
 gives (integer results: the tolerance is zero) on two calls in a row that share the array,
-and that it refuses a problem whose lowered matrix does not fit.
+that both equal the CPU oracle's direct convolution, and that it refuses a problem whose
+lowered matrix does not fit.
 
 The file name makes pytest collect it after every other test file.
 """
@@ -14,7 +15,9 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import oracle as orc
 from paper_1709_04060_b200 import synth
+from qnn_testutil import decode_out
 
 pytestmark = pytest.mark.gpu
 
@@ -80,6 +83,26 @@ def test_two_calls_in_a_row_match_qconv(qb, fmt):
         assert np.array_equal(got, want)
         want_raw, got_raw = _both(qb, d, Wp, x, None)          # raw int32 accumulators
         assert np.array_equal(got_raw, want_raw)
+        # and against the oracle's direct convolution (codes and accumulators)
+        npix = case.B * case.OH * case.OW
+        ref = orc.qconv(case.In, case.Wt, case.thr, case.stride, case.pad).reshape(npix, case.OC)
+        assert np.array_equal(decode_out(got, INT8, case.out_bits, npix, case.OC, False), ref)
+        ref_acc = orc.conv_direct(case.In, case.Wt, case.stride, case.pad).reshape(npix, case.OC)
+        assert np.array_equal(decode_out(got_raw, INT8, 0, npix, case.OC, True), ref_acc)
+
+
+@pytest.mark.parametrize("C", [3, 5, 20])
+def test_bipolar_weights_small_channel_counts(qb, C):
+    """Bipolar (+-1) filters over an 8-bit map whose channel count is not a multiple of 16:
+    the pad columns of the packed weight rows are -1, not 0, so the result depends on the
+    lowered matrix being zero there.  Against the oracle and against qnn_qconv."""
+    case = synth.conv_case(40 + C, 2, 14, 13, C, 24, 3, 3, 1, 0, 1, 2)
+    d, Wp, x, thr = _setup(qb, case, INT8)
+    want, got = _both(qb, d, Wp, x, thr)
+    assert np.array_equal(got, want)
+    npix = case.B * case.OH * case.OW
+    ref = orc.qconv(case.In, case.Wt, case.thr, case.stride, case.pad).reshape(npix, case.OC)
+    assert np.array_equal(decode_out(got, INT8, case.out_bits, npix, case.OC, False), ref)
 
 
 def test_problem_larger_than_the_array_is_refused(qb):
