@@ -146,6 +146,208 @@ def run_reference(args):
     }))
 
 
+def oracle_other_configs():
+    """The oracle as it stands on the other configurations (or a bounded sample of them):
+    config 1 in full, one conv2-shaped image, one AlexNet-shaped image, config 5 at N = 1."""
+    from oracle import oracle as orc, alexnet as onet
+    from paper_1709_04060_b200 import synth
+    res = {}
+    c1 = synth.gemm_case(1, 64, 256, 576, 1, 2)
+    orc.qgemm(c1.W, c1.At, c1.thr)
+    t0 = time.perf_counter()
+    for _ in range(20):
+        orc.qgemm(c1.W, c1.At, c1.thr)
+    dt = (time.perf_counter() - t0) / 20
+    res["config1"] = {"us": 1e6 * dt, "mac_per_s": 64 * 256 * 576 / dt, "sample": "the whole problem, mean of 20"}
+    c3 = synth.conv2_alexnet_case(1)
+    t0 = time.perf_counter()
+    orc.qconv(c3.In, c3.Wt, c3.thr, c3.stride, c3.pad)
+    dt = time.perf_counter() - t0
+    res["config3"] = {"images_per_s": 1.0 / dt, "mac_per_s": 729 * 256 * 2400 / dt, "sample": "one image (direct convolution)"}
+    net = synth.alexnet_case(1)
+    t0 = time.perf_counter()
+    onet.forward(net, keep_intermediates=False)
+    dt = time.perf_counter() - t0
+    res["config4"] = {"images_per_s": 1.0 / dt, "mac_per_s": 1.135e9 / dt, "sample": "one image through the whole chain"}
+    c5 = synth.gemm_case(5021, 8192, 1, 8192, 2, 2)
+    t0 = time.perf_counter()
+    orc.qgemm(c5.W, c5.At, c5.thr)
+    dt = time.perf_counter() - t0
+    res["config5"] = {"us": 1e6 * dt, "mac_per_s": 8192 * 8192 / dt, "sample": "W2A2, N = 1, the whole problem"}
+    res["cores"] = orc.num_threads()
+    return res
+
+
+def sustained_mma_peak(torch, qb, seconds=1.5):
+    """The widest CTA-pair MMA issued back to back for `seconds`: the int8 tensor peak the GPU
+    holds under its power cap (TOP/s), i.e. the denominator for kernels timed inside a long loop."""
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    st, ops = qb.qnn_peak_mma_i8(1, 256, 65536)         # ~4.6 ms per launch
+    qb.check(st)
+    torch.cuda.synchronize()
+    n = max(1, int(seconds / 4.6e-3))
+    e0.record()
+    for _ in range(n):
+        qb.check(qb.qnn_peak_mma_i8(1, 256, 65536)[0])
+    e1.record()
+    torch.cuda.synchronize()
+    return round(n * ops / (e0.elapsed_time(e1) * 1e-3) / 1e12, 1)
+
+
+def roofline_entry(achieved_tops, gemm_avg_ms, timed_seconds, clocks, peaks, measured):
+    """Tensor roofline of the dominant kernel.  The denominator is the int8 MMA issue rate measured
+    in this run: the sustained figure when the timed region ran for a second or more under the
+    power cap, else the burst figure; the other candidates are printed beside it."""
+    long_run = timed_seconds >= 1.0 or (clocks and "sw_power_cap" in (clocks.get("reasons") or []))
+    cands = {"2x_bf16_cublas_sustained_of_" + peaks["source"]: 2.0 * peaks["bf16_sustained"],
+             "2x_bf16_cublas_burst_of_" + peaks["source"]: 2.0 * peaks["bf16_burst"],
+             "nominal_dense_int8": 4500.0}
+    if measured:
+        cands["int8_mma_burst_measured"] = measured["mma_i8"]["mode1_n256"]
+        cands["int8_mma_sustained_measured"] = measured["mma_i8_sustained"]
+        key = "int8_mma_sustained_measured" if long_run else "int8_mma_burst_measured"
+    else:
+        key = "2x_bf16_cublas_sustained_of_" + peaks["source"] if long_run else "2x_bf16_cublas_burst_of_" + peaks["source"]
+    peak = cands[key]
+    return {"bound": "tensor", "achieved": achieved_tops, "peak": peak, "unit": "TOP/s",
+            "frac": achieved_tops / peak, "peak_source": key,
+            "frac_vs": {k: round(achieved_tops / v, 3) for k, v in cands.items()},
+            "peaks_tops": cands,
+            "traffic": TRAFFIC_BYTES_PER_LAUNCH,
+            "traffic_source": "ncu dram__bytes of one 4096^3 W1A2 launch (constant from that capture)",
+            "kernel": "qgemm_tc2_kernel (CTA-pair tcgen05 kernel, 4096^3, int8 operands)",
+            "avg_launch_ms": gemm_avg_ms, "algorithmic_ops_per_launch": 2.0 * DIM ** 3}
+
+
+def measure_other_configs(torch, qb, synth, peaks, measured):
+    """Configurations 1, 3, 4 (per layer) and 5 in compact form, each with the roofline that
+    bounds it: latency for the small GEMM, HBM for lowering and the few-column fully connected
+    layers (weights rotated through more than twice the L2 size), tensor for the rest."""
+    from paper_1709_04060_b200.alexnet import AlexNetPlan
+    PL, I8 = qb.QNN_FMT_BITPLANES, qb.QNN_FMT_INT8
+    hbm = peaks["hbm_gbs"]
+    tpeak = measured["mma_i8"]["mode1_n256"]             # burst: these kernels are timed in short loops
+    res = {"hbm_peak_gbs": hbm, "tensor_peak_tops": tpeak, "peak_source": f"HBM: {peaks['source']} copy; tensor: int8 MMA burst measured in this run"}
+
+    # config 1: one small W1A2 GEMM + threshold (launch-latency bound)
+    c = synth.gemm_case(1, 64, 256, 576, 1, 2)
+    row = {}
+    for fmt, name in ((I8, "int8"), (PL, "bitplanes")):
+        Wp = qb.pack(qb.to_device_logical(c.W, c.w_enc), 1, c.w_enc, fmt)
+        Ap = qb.pack(qb.to_device_logical(c.At, c.a_enc), 2, c.a_enc, fmt)
+        thr = torch.from_numpy(c.thr).cuda()
+        d = qb.gemm_desc(64, 256, 576, 1, 2, 2, c.w_enc, c.a_enc, fmt, I8)
+        out = torch.empty(qb.qnn_gemm_out_bytes(d, True), dtype=torch.uint8, device="cuda")
+        ms = _time_calls(torch, lambda i: qb.check(qb.qnn_qgemm(d, Wp, Ap, thr, out)), 50, graph=True)
+        row[name + "_us"] = round(1e3 * ms, 2)
+    row.update({"bound": "latency", "mac": 64 * 256 * 576, "gmacs_int8": round(64 * 256 * 576 / row["int8_us"] / 1e3, 1)})
+    res["config1"] = row
+
+    # config 3: conv2-shaped W1A2 layer, 8-bit maps: explicit lowering (HBM) and the whole layer (tensor)
+    conv = {}
+    for B in (1, 64):
+        c = synth.conv2_alexnet_case(B)
+        x = torch.from_numpy(c.In.astype(np.uint8)).cuda()
+        Wp = qb.pack(qb.to_device_logical(c.Wt.reshape(c.OC, -1), c.w_enc), 1, c.w_enc, I8)
+        d = qb.qnn_conv_desc(B, 27, 27, 96, 96, 256, 5, 5, 1, 2, 1, 2, 2, c.w_enc, c.a_enc, I8, I8, 0)
+        thr = torch.from_numpy(c.thr).cuda()
+        ws = torch.empty(qb.qnn_conv_workspace_bytes(d), dtype=torch.uint8, device="cuda")
+        out = torch.empty(qb.qnn_conv_out_bytes(d, True), dtype=torch.uint8, device="cuda")
+        ms_low = _time_calls(torch, lambda i: qb.check(qb.qnn_im2col(d, x, ws)), 20, graph=True)
+        ms_all = _time_calls(torch, lambda i: qb.check(qb.qnn_qconv(d, Wp, x, thr, out, ws, ws.numel())), 20, graph=True)
+        low_bytes = qb.qnn_conv_lowered_bytes(d) + x.numel()
+        macs = B * 729 * 256 * 2400
+        conv[f"B{B}"] = {"im2col_us": round(1e3 * ms_low, 2), "im2col_gbs": round(low_bytes / ms_low / 1e6, 1),
+                         "im2col_hbm_frac": round(low_bytes / ms_low / 1e6 / hbm, 3),
+                         "qconv_us": round(1e3 * ms_all, 2), "images_per_s": round(B / ms_all * 1e3, 1),
+                         "tmacs": round(macs / ms_all / 1e9, 1), "tensor_frac": round(2 * macs / ms_all / 1e9 / tpeak, 3)}
+        del ws, out
+    conv["note"] = "lowered matrix of B = 1 (1.75 MB) stays in L2; B = 64 (112 MB) is close to the L2 size"
+    res["config3"] = conv
+
+    # config 5: M = K = 8192; few columns (HBM bound, packed bytes) and N = 8192 (tensor bound)
+    M = K = 8192
+    skinny = []
+    for bits in (2, 4):
+        c = synth.gemm_case(5000 + bits, M, 16, K, bits, bits)
+        Wd = qb.to_device_logical(c.W, c.w_enc)
+        thr = torch.from_numpy(c.thr).cuda()
+        packed_bytes = M * K * bits // 8
+        for wfmt, afmt, name in SKINNY_FORMATS(qb):
+            Wp = qb.pack(Wd, bits, c.w_enc, wfmt)
+            copies = max(2, int(300e6 // Wp.numel()) + 1)          # > 2 x L2 in rotation
+            Wrot = [Wp] + [Wp.clone() for _ in range(copies - 1)]
+            for N in (1, 4, 16):
+                Ap = qb.pack(qb.to_device_logical(c.At[:N], c.a_enc), bits, c.a_enc, afmt)
+                d = qb.qnn_gemm_desc(M, N, K, bits, bits, bits, c.w_enc, c.a_enc, wfmt, afmt, I8, 0)
+                out = torch.empty(qb.qnn_gemm_out_bytes(d, True), dtype=torch.uint8, device="cuda")
+                ms = _time_calls(torch, lambda i: qb.check(qb.qnn_qgemm(d, Wrot[i % copies], Ap, thr, out)),
+                                 2 * copies, graph=True)
+                alg = packed_bytes + N * K * bits // 8 + thr.numel() * 4 + N * M
+                skinny.append({"w": bits, "a": bits, "N": N, "fmt": name, "us": round(1e3 * ms, 2),
+                               "gbs_packed": round(alg / ms / 1e6, 1), "hbm_frac_packed": round(alg / ms / 1e6 / hbm, 3),
+                               "bytes_read_per_call": Wp.numel() + Ap.numel() + thr.numel() * 4})
+            del Wrot, Wp
+    res["config5_skinny"] = {"rows": skinny, "bound": "hbm",
+                             "note": "hbm_frac_packed = bytes of the w-bit packed problem (weights w*M*K/8, activations, "
+                                     "thresholds, codes) / time / HBM peak, whatever operand format the kernel reads"}
+    sets = [(torch.randint(-2, 2, (M, K), dtype=torch.int8, device="cuda"),
+             torch.randint(0, 4, (M, K), dtype=torch.uint8, device="cuda")) for _ in range(2)]
+    thr_l = torch.sort(torch.randint(-300, 300, (M, 3), dtype=torch.int32, device="cuda"), dim=1).values.contiguous()
+    out_l = torch.empty(M * M, dtype=torch.uint8, device="cuda")
+    dl = qb.gemm_desc(M, M, K, 2, 2, 2, qb.QNN_ENC_SIGNED, qb.QNN_ENC_UNSIGNED, I8, I8)
+    ms_l = _time_calls(torch, lambda i: qb.check(qb.qnn_qgemm(dl, sets[i % 2][0], sets[i % 2][1], thr_l, out_l)), 6, graph=True)
+    res["config5_n8192"] = {"us": round(1e3 * ms_l, 1), "tmacs": round(M ** 3 / ms_l / 1e9, 1),
+                            "tensor_frac": round(2 * M ** 3 / ms_l / 1e9 / tpeak, 3), "bound": "tensor"}
+    del sets, out_l
+
+    # config 4: per-layer times of the AlexNet-shaped chain at batch 256
+    B = 256
+    net = synth.alexnet_case(B)
+    plan = AlexNetPlan(net, B, "auto")
+    img = torch.from_numpy(net.image.astype(np.uint8)).cuda()
+    plan.forward(img)
+    per_layer, prev, total_us = {}, None, 0.0
+    macs = {"conv1": 1.054e8, "conv2": 4.479e8, "conv3": 1.495e8, "conv4": 2.243e8, "conv5": 1.495e8,
+            "fc6": 3.77e7, "fc7": 1.68e7, "fc8": 4.10e6}
+    for (kind, d, Wp, thr, out), name in zip(plan.steps, plan.names):
+        x_in = img if prev is None else prev
+        if kind == "conv":
+            f = lambda i: qb.check(qb.qnn_qconv(d, Wp, x_in, thr, out, plan.workspace, plan.workspace.numel()))
+        elif kind == "pool":
+            f = lambda i: qb.check(qb.qnn_maxpool(d, x_in, out))
+        else:
+            f = lambda i: qb.check(qb.qnn_qgemm(d, Wp, x_in, thr, out, None, 0))
+        us = 1e3 * _time_calls(torch, f, 10, graph=True)
+        entry = {"us": round(us, 1)}
+        if name in macs:
+            entry["tensor_frac"] = round(2 * macs[name] * B / us / 1e6 / tpeak, 3)
+        else:
+            nbytes = x_in.numel() + out.numel()
+            entry["gbs"] = round(nbytes / us / 1e3, 1)
+            entry["hbm_frac"] = round(nbytes / us / 1e3 / hbm, 3)
+        per_layer[name] = entry
+        total_us += us
+        prev = out
+    matrix_us = sum(v["us"] for k, v in per_layer.items() if k in macs)
+    res["config4_batch256_layers"] = {"per_layer": per_layer, "sum_us": round(total_us, 1),
+                                      "share_8bit_layers": round((per_layer["conv1"]["us"] + per_layer["fc8"]["us"]) / total_us, 3),
+                                      "share_matrix_layers": round(matrix_us / total_us, 3),
+                                      "chain_tensor_frac": round(2 * 1.135e9 * B / total_us / 1e6 / tpeak, 3)}
+    st, dev = qb.qnn_device_status()
+    assert st == 0 and dev == 0
+    return res
+
+
+def SKINNY_FORMATS(qb):
+    """(weight format, activation format, label) triples the few-column benchmark runs."""
+    PL, I8 = qb.QNN_FMT_BITPLANES, qb.QNN_FMT_INT8
+    fmts = [(PL, PL, "bitplanes"), (I8, I8, "int8")]
+    if hasattr(qb, "QNN_FMT_FIELDS"):
+        fmts.insert(0, (qb.QNN_FMT_FIELDS, I8, "fields"))
+    return fmts
+
+
 def run_b200(args):
     import torch
     from paper_1709_04060_b200 import dist as qdist, synth
@@ -255,7 +457,6 @@ def run_b200(args):
     gemm_ms = [a.elapsed_time(b) for (a, b) in gemm_events]
     gemm_avg_ms = float(np.mean(gemm_ms))
     achieved_tops = 2.0 * DIM ** 3 / (gemm_avg_ms * 1e-3) / 1e12
-    tensor_peak = 2.0 * peaks["bf16_sustained"]
     per_pair = {}
     for i, (w, a) in enumerate(PAIRS):
         t = float(np.mean(gemm_ms[i::len(PAIRS)]))
@@ -287,7 +488,16 @@ def run_b200(args):
         m, s, threads = oracle_sample_run(rows, pairs)
         cpu = {"value": m / s, "unit": UNIT, "cores": threads, "kind": "oracle",
                "sample": f"first {rows} weight rows x all {DIM} columns, K={DIM}, (w,a) in {pairs}: "
-                         f"{m:.3g} MAC in {s:.1f} s"}
+                         f"{m:.3g} MAC in {s:.1f} s",
+               "other_configs": oracle_other_configs()}
+
+    # ---- roofline denominators measured in this run, and the other configurations
+    measured = other = None
+    if world == 1:
+        measured = measure_peaks(torch, qb, ((1, 256), (0, 256)), mmas=8192, popc_iters=8192, reps=3)
+        measured["mma_i8_sustained"] = sustained_mma_peak(torch, qb, seconds=1.5)
+        if not args.no_other_configs:
+            other = measure_other_configs(torch, qb, synth, peaks, measured)
 
     # ---- second half of the metric: AlexNet-shaped W1A2 chain, images/s (N = 1 only)
     alexnet = None
@@ -303,6 +513,9 @@ def run_b200(args):
             alexnet[f"batch{B}"] = {"images_per_s": B / ms_b * 1e3, "ms": ms_b,
                                     "kernels_per_forward": plan.launches_per_forward()}
             del graph, plan
+        if cpu is not None:
+            alexnet["oracle_images_per_s_batch1"] = cpu["other_configs"]["config4"]["images_per_s"]
+            alexnet["oracle_cores"] = cpu["other_configs"]["cores"]
         alexnet["note"] = ("random-init AlexNet-shaped W1A2 chain (conv1/fc8 8-bit), uint8 images resident "
                            "in HBM, one CUDA-graph replay per forward pass")
 
@@ -320,14 +533,11 @@ def run_b200(args):
                 "h2d_bytes_per_step": len(PAIRS) * DIM * DIM, "d2h_bytes_per_step": len(PAIRS) * DIM * DIM,
                 "steps": e2e_steps},
         "gpu_launches": int(launches),
-        "roofline": {"bound": "tensor", "achieved": achieved_tops, "peak": tensor_peak, "unit": "TOP/s",
-                     "frac": achieved_tops / tensor_peak,
-                     "traffic": TRAFFIC_BYTES_PER_LAUNCH,
-                     "kernel": "qgemm_tc2_kernel (CTA-pair tcgen05 kernel, 4096^3, int8 operands)",
-                     "peak_source": f"2 x {peaks['source']} bf16 sustained cuBLAS TFLOP/s (nominal int8:bf16 ratio)",
-                     "avg_launch_ms": gemm_avg_ms, "algorithmic_ops_per_launch": 2.0 * DIM ** 3},
+        "roofline": roofline_entry(achieved_tops, gemm_avg_ms, ms * 1e-3, clocks, peaks, measured),
         "per_pair_tmacs": per_pair,
+        "measured_peaks": measured,
         "alexnet_w1a2": alexnet,
+        "other_configs": other,
         "cpu_baseline": cpu,
     }
     print(json.dumps(out))
@@ -372,7 +582,8 @@ def _time_calls(torch, fn, iters, warmup=3, graph=False):
 def measure_peaks(torch, qb, mma_configs=((1, 256),), mmas=4096, popc_iters=4096, reps=5):
     """Issue-bound peaks of the two GEMM paths, timed with CUDA events (best of `reps`):
     tcgen05 kind::i8 MMAs on shared-memory-resident tiles (pair: cta_group::2) and XOR+POPC
-    chains.  Returns {"mma_i8": {"pair<p>_n<n>": TOP/s, ...}, "popc_g_per_s": ..}."""
+    chains.  Returns {"mma_i8": {"mode<m>_n<n>": TOP/s, ...}, "popc_g_per_s": ..}; mode 0: one CTA per
+    SM, 1: CTA pairs, 2: one CTA per SM with the 128-row operand in tensor memory."""
     out = {"mma_i8": {}}
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for (pair, n) in mma_configs:
@@ -386,7 +597,7 @@ def measure_peaks(torch, qb, mma_configs=((1, 256),), mmas=4096, popc_iters=4096
             if r > 0:
                 ms = e0.elapsed_time(e1)
                 best = ms if best is None else min(best, ms)
-        out["mma_i8"][f"pair{pair}_n{n}"] = round(ops / (best * 1e-3) / 1e12, 1)
+        out["mma_i8"][f"mode{pair}_n{n}"] = round(ops / (best * 1e-3) / 1e12, 1)
     sink = torch.empty(qb.qnn_peak_popc_sink_bytes(), dtype=torch.uint8, device="cuda")
     best = None
     for r in range(reps + 1):
@@ -418,19 +629,20 @@ def run_peaks(args):
     sampler.start()
     time.sleep(0.15)
     t0 = time.time()
-    cfgs = [(0, n) for n in (16, 32, 64, 128, 256)] + [(1, n) for n in (32, 64, 128, 256)]
+    cfgs = ([(0, n) for n in (16, 32, 64, 128, 256)] + [(1, n) for n in (32, 64, 128, 256)] +
+            [(2, n) for n in (16, 32, 64, 128)])          # mode 2: 128-row operand from tensor memory
     res = measure_peaks(torch, qb, cfgs, mmas=16384, popc_iters=16384, reps=8)
     # a seconds-long run of the widest pair MMA: the sustained figure under the power cap
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     total = 0.0
-    for _ in range(60):
+    for _ in range(400):
         st, ops = qb.qnn_peak_mma_i8(1, 256, 65536)
         qb.check(st)
         total += ops
     e1.record()
     torch.cuda.synchronize()
-    res["mma_i8_sustained_pair1_n256"] = round(total / (e0.elapsed_time(e1) * 1e-3) / 1e12, 1)
+    res["mma_i8_sustained_mode1_n256"] = round(total / (e0.elapsed_time(e1) * 1e-3) / 1e12, 1)
     res["sustained_seconds"] = round(e0.elapsed_time(e1) * 1e-3, 2)
     clocks = sampler.stop(t0, time.time())
     peaks = load_peaks()
@@ -612,8 +824,8 @@ def run_shapes(args):
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one 4096^3 W1A2 launch of the (CTA-pair)
-# tensor-core kernel, from the ncu capture summarised in profiles/qgemm_tc2_4096_w1a2_w4a4.md (the output
-# codes were still in L2 when the capture ended, so the write counter is small).
+# tensor-core kernel, from an ncu capture of that launch (the output codes were still in L2 when
+# the capture ended, so the write counter is small).
 TRAFFIC_BYTES_PER_LAUNCH = 33648384 + 79360
 
 
@@ -625,6 +837,8 @@ def main():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-alexnet", action="store_true", help="skip the AlexNet-shaped chain measurement")
+    ap.add_argument("--no-other-configs", action="store_true",
+                    help="skip the compact measurements of configurations 1, 3, 4 (per layer) and 5")
     ap.add_argument("--overlap", type=int, default=1,
                     help="1: activation packer on a second stream, overlapping the previous GEMM (default); 0: one stream")
     ap.add_argument("--extras-only", default=None, choices=["large", "skinny", "conv2", "alexnet"],

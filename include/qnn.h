@@ -259,14 +259,15 @@ qnn_status qnn_streamline(const qnn_channel_params *ch, int channels, const doub
 
 /* ---- roofline denominators (Section 4.1.1 reports against the machine's peak) -- */
 
-/* Launches the tensor-pipe issue-rate microbenchmark on `stream`: every SM (pair == 0; one
- * CTA each) or every pair of SMs (pair != 0; tcgen05 cta_group::2) issues mmas_per_cta
+/* Launches the tensor-pipe issue-rate microbenchmark on `stream`: every SM (mode 0; one
+ * CTA each; mode 2: the same with the 128-row operand read from tensor memory, n <= 128) or
+ * every pair of SMs (mode 1; tcgen05 cta_group::2) issues mmas_per_cta
  * back-to-back tcgen05.mma kind::i8 instructions of 128 (256 for a pair) x n x 32 on operand
- * tiles resident in shared memory: no loads, no epilogue.  n: a multiple of 16 (32 for a
- * pair) in [16, 256].  *ops (host) receives the integer operations (2 per multiply-
+ * tiles of pseudo-random bytes resident in shared memory: no loads, no epilogue.  n: a
+ * multiple of 16 (32 for a pair) in [16, 256].  *ops (host) receives the integer operations (2 per multiply-
  * accumulate) the launch performs; the caller times the launch with events.  The peak of
  * the dense int8 tensor path is ops / time.  Errors: INVALID_ARG, CUDA. */
-qnn_status qnn_peak_mma_i8(int pair, int n, int mmas_per_cta, double *ops, void *stream);
+qnn_status qnn_peak_mma_i8(int mode, int n, int mmas_per_cta, double *ops, void *stream);
 
 /* Launches the POPC issue-rate microbenchmark (chains of XOR + POPC in registers, the inner
  * operation of Algorithm 1): *popcs (host) receives the number of 32-bit population counts

@@ -3,7 +3,8 @@
 // throughput, Section 4.1.1; these are the same two peaks for this GPU):
 //
 //  * tensor path:  tcgen05.mma kind::i8 issued back to back on operand tiles that already sit in
-//    shared memory -- no loads, no epilogue, nothing to wait for but the tensor pipe itself;
+//    shared memory (or, for the 128-row operand, in tensor memory) -- no loads, no epilogue,
+//    nothing to wait for but the tensor pipe itself;
 //  * bit-serial path: chains of XOR + POPC, the inner operation of Algorithm 1, in registers.
 //
 // Both kernels touch no global memory besides one result word per thread (POPC) and are timed
@@ -24,19 +25,37 @@ struct PeakSmem {
     int abort_flag;
 };
 
-// PAIR == false: every CTA issues `mmas` MMAs of 128 x n x 32; PAIR == true: the leader of every
-// CTA pair issues `mmas` MMAs of 256 x n x 32 (cta_group::2) that read both CTAs' tiles.
-template <bool PAIR>
+// A operand (128 rows x 32 depth bytes) taken from tensor memory instead of shared memory.
+__device__ __forceinline__ void umma_i8_tmem_a(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+enum { PK_SINGLE = 0, PK_PAIR = 1, PK_TMEM_A = 2 };
+
+// MODE PK_SINGLE: every CTA issues `mmas` MMAs of 128 x n x 32; PK_PAIR: the leader of every CTA
+// pair issues `mmas` MMAs of 256 x n x 32 (cta_group::2) that read both CTAs' tiles; PK_TMEM_A: as
+// PK_SINGLE with the 128-row operand read from tensor memory.
+template <int MODE>
 __global__ void __launch_bounds__(128, 1) peak_mma_i8_kernel(int n, int mmas, int *status_word) {
+    constexpr bool PAIR = MODE == PK_PAIR;
     extern __shared__ uint8_t pk_raw[];
     PeakSmem &sm = *reinterpret_cast<PeakSmem *>(pk_raw + ((1024u - (smem_u32(pk_raw) & 1023u)) & 1023u));
     const int warp = threadIdx.x >> 5;
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
     volatile int *abort_flag = &sm.abort_flag;
 
-    // operand values do not matter for the rate; zeros keep the accumulators at zero
-    for (int i = threadIdx.x; i < (int)(sizeof(sm.a) / 16); i += blockDim.x) reinterpret_cast<uint4 *>(sm.a)[i] = make_uint4(0, 0, 0, 0);
-    for (int i = threadIdx.x; i < (int)(sizeof(sm.b) / 16); i += blockDim.x) reinterpret_cast<uint4 *>(sm.b)[i] = make_uint4(0, 0, 0, 0);
+    // operand values do not change the instruction rate, but they do change the power drawn (and
+    // with it the clock under the power cap): pseudo-random bytes, as a real GEMM would see; the
+    // int32 accumulators simply wrap
+    uint32_t h = 0x9E3779B9u * (uint32_t)(blockIdx.x * blockDim.x + threadIdx.x + 1);
+    for (int i = threadIdx.x; i < (int)((sizeof(sm.a) + sizeof(sm.b)) / 4); i += blockDim.x) {
+        h = h * 1664525u + 1013904223u;
+        reinterpret_cast<uint32_t *>(sm.a)[i] = h ^ (h >> 15);        // a and b are adjacent
+    }
     if (threadIdx.x == 0) {
         mbar_init(&sm.done, 1);
         sm.abort_flag = 0;
@@ -59,8 +78,10 @@ __global__ void __launch_bounds__(128, 1) peak_mma_i8_kernel(int n, int mmas, in
             const int st = (i >> 2) % PK_STAGES, kk = i & 3;
             const uint64_t da = umma_smem_desc(smem_u32(sm.a[st])) + 2 * kk;
             const uint64_t db = umma_smem_desc(smem_u32(sm.b[st])) + 2 * kk;
-            const uint32_t d = tmem_base + (uint32_t)(((i >> 7) & 1) * 256);      // two accumulators, 128 MMAs each in turn
+            // two accumulators, 128 MMAs each in turn (PK_TMEM_A: n <= 128, columns 384.. hold the operand)
+            const uint32_t d = tmem_base + (uint32_t)(((i >> 7) & 1) * (MODE == PK_TMEM_A ? 128 : 256));
             if (PAIR) umma_i8_pair(d, da, db, idesc, 1u);
+            else if (MODE == PK_TMEM_A) umma_i8_tmem_a(d, tmem_base + 384u + (uint32_t)(8 * (i & 7)), db, idesc, 1u);
             else umma_i8(d, da, db, idesc, 1u);
         }
         if (PAIR) umma_commit_pair(map_to_cta(smem_u32(&sm.done), 0));
@@ -103,21 +124,25 @@ using namespace qnn;
 
 extern "C" {
 
-qnn_status qnn_peak_mma_i8(int pair, int n, int mmas_per_cta, double *ops, void *stream) {
-    if (!ops || mmas_per_cta <= 0 || n < 16 || n > 256 || (n % 16) != 0 || (pair && (n % 32) != 0))
+qnn_status qnn_peak_mma_i8(int mode, int n, int mmas_per_cta, double *ops, void *stream) {
+    if (!ops || mmas_per_cta <= 0 || n < 16 || n > 256 || (n % 16) != 0 || mode < 0 || mode > 2 ||
+        (mode == PK_PAIR && (n % 32) != 0) || (mode == PK_TMEM_A && n > 128))
         return QNN_ERR_INVALID_ARG;
+    const bool pair = mode == PK_PAIR;
     int *status = device_status_word();
     if (!status) return QNN_ERR_CUDA;
     const int sms = sm_count();
     const size_t smem = sizeof(PeakSmem) + 1024;
     const int dev = current_device();
     if (dev < 0) return QNN_ERR_CUDA;
-    static bool attr_done[2][QNN_MAX_DEVICES] = {{false}};
-    if (!attr_done[pair ? 1 : 0][dev]) {
-        const cudaError_t e = pair ? cudaFuncSetAttribute(peak_mma_i8_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
-                                   : cudaFuncSetAttribute(peak_mma_i8_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return QNN_ERR_CUDA;
-        attr_done[pair ? 1 : 0][dev] = true;
+    static bool attr_done[3][QNN_MAX_DEVICES] = {{false}};
+    if (!attr_done[mode][dev]) {
+        const void *fn = mode == PK_PAIR ? (const void *)peak_mma_i8_kernel<PK_PAIR>
+                         : (mode == PK_TMEM_A ? (const void *)peak_mma_i8_kernel<PK_TMEM_A>
+                                              : (const void *)peak_mma_i8_kernel<PK_SINGLE>);
+        if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return QNN_ERR_CUDA;
+        attr_done[mode][dev] = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = smem; cfg.stream = (cudaStream_t)stream;
@@ -129,11 +154,12 @@ qnn_status qnn_peak_mma_i8(int pair, int n, int mmas_per_cta, double *ops, void 
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
         cfg.numAttrs = 1;
-        e = cudaLaunchKernelEx(&cfg, peak_mma_i8_kernel<true>, n, mmas_per_cta, status);
+        e = cudaLaunchKernelEx(&cfg, peak_mma_i8_kernel<PK_PAIR>, n, mmas_per_cta, status);
         *ops = 2.0 * 256.0 * n * 32.0 * (double)mmas_per_cta * (sms / 2);
     } else {
         cfg.gridDim = dim3(sms);
-        e = cudaLaunchKernelEx(&cfg, peak_mma_i8_kernel<false>, n, mmas_per_cta, status);
+        e = mode == PK_TMEM_A ? cudaLaunchKernelEx(&cfg, peak_mma_i8_kernel<PK_TMEM_A>, n, mmas_per_cta, status)
+                              : cudaLaunchKernelEx(&cfg, peak_mma_i8_kernel<PK_SINGLE>, n, mmas_per_cta, status);
         *ops = 2.0 * 128.0 * n * 32.0 * (double)mmas_per_cta * sms;
     }
     if (e != cudaSuccess) return QNN_ERR_CUDA;
