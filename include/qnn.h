@@ -47,6 +47,19 @@
  *                      uint8 for UNSIGNED (the 8-bit formulation of Section 3:
  *                      few-bit values held in 8-bit containers); the tensor-core
  *                      path consumes this.
+ *   QNN_FMT_FIELDS     weights only: w-bit fields packed along the depth, f = 1, 2 or 4
+ *                      bits per field (3-bit values take 4-bit fields), S = 8/f fields
+ *                      per byte, [rows][ldf] bytes with ldf = 32 * ceil(K / (32 S)).
+ *                      Element k of a row lies in byte 32 g + j at bits [f s, f s + f),
+ *                      where g = k / (32 S), s = (k mod 32 S) / 32, j = k mod 32: the 32
+ *                      elements at field position s of 32 consecutive bytes are 32
+ *                      consecutive depth indices.  A field holds the value minus the
+ *                      encoding's minimum (UNSIGNED: the value, SIGNED: value + 2^(b-1),
+ *                      BIPOLAR: the bit); fields past K are zero.  This is the paper's
+ *                      packed weight storage (Section 4.2: fully connected layers gain
+ *                      from the cut in memory traffic) in a form that expands to 8-bit
+ *                      values with one AND per word; qnn_qgemm takes it with INT8
+ *                      activations and N <= 16 columns.
  */
 #ifndef QNN_H_
 #define QNN_H_
@@ -69,7 +82,7 @@ typedef enum {
 } qnn_status;
 
 typedef enum { QNN_ENC_UNSIGNED = 0, QNN_ENC_SIGNED = 1, QNN_ENC_BIPOLAR = 2 } qnn_enc;
-typedef enum { QNN_FMT_BITPLANES = 0, QNN_FMT_INT8 = 1 } qnn_fmt;
+typedef enum { QNN_FMT_BITPLANES = 0, QNN_FMT_INT8 = 1, QNN_FMT_FIELDS = 2 } qnn_fmt;
 typedef enum { QNN_PATH_AUTO = 0, QNN_PATH_BITSERIAL = 1, QNN_PATH_TCGEN05_I8 = 2 } qnn_path;
 
 /* ---- packer (Section 3.1 bit planes; Section 3 8-bit containers) ---------- */
@@ -79,11 +92,12 @@ typedef struct {
     int K;           /* depth                                                 */
     int bits;        /* 1..8; BIPOLAR requires 1                              */
     int enc;         /* qnn_enc                                               */
-    int fmt;         /* qnn_fmt of the packed result                          */
+    int fmt;         /* qnn_fmt of the packed result (FIELDS: bits <= 4)      */
 } qnn_pack_desc;
 
 /* Row pitch of a packed operand: 32-bit words per row and plane for BITPLANES
- * (ceil(K/32)), bytes per row for INT8 (K rounded up to 16).  Host only. */
+ * (ceil(K/32)), bytes per row for INT8 (K rounded up to 16); 0 for FIELDS, whose pitch
+ * depends on the bit width (qnn_packed_bytes / rows).  Host only. */
 size_t qnn_packed_ld(int K, int fmt);
 
 /* Bytes of a packed operand.  Host only; 0 on invalid arguments. */
@@ -103,7 +117,8 @@ typedef struct {
     int out_bits;         /* 1..4: 2^out_bits - 1 thresholds per row; ignored
                              when thr == NULL                                 */
     int w_enc, a_enc;     /* qnn_enc                                          */
-    int w_fmt, a_fmt;     /* qnn_fmt; both operands must use the same format  */
+    int w_fmt, a_fmt;     /* qnn_fmt; both operands must use the same format,
+                             except w_fmt FIELDS, which goes with a_fmt INT8     */
     int out_fmt;          /* qnn_fmt of the output codes; ignored if thr==NULL*/
     int path;             /* qnn_path; AUTO selects by operand format, and for a
                              handful of columns (N <= 16 bit planes, N <= 8
@@ -125,8 +140,11 @@ size_t qnn_gemm_out_bytes(const qnn_gemm_desc *d, int has_thresholds);
  *   out_fmt BITPLANES  uint32 [out_bits][N][ceil(M/32)], pad bits 0
  *   thr == NULL        int32  [N][M] raw accumulators
  * The accumulators never reach global memory on the fused path.
+ * w_fmt FIELDS (with a_fmt INT8): N <= 16, w_bits <= 4; the packed weights are read
+ * from memory once and expanded inside the kernel.
  * Errors: INVALID_ARG, UNSUPPORTED (mixed formats, bits out of range for the
- * path, BIPOLAR with bits != 1), ALIGNMENT, WORKSPACE, CUDA. */
+ * path, BIPOLAR with bits != 1, FIELDS with more than 16 columns or a depth slice that
+ * does not fit shared memory), ALIGNMENT, WORKSPACE, CUDA. */
 qnn_status qnn_qgemm(const qnn_gemm_desc *d, const void *W, const void *A,
                      const int32_t *thr, void *out,
                      void *workspace, size_t workspace_bytes, void *stream);

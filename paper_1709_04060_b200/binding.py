@@ -28,7 +28,7 @@ QNN_OK = 0
 QNN_ERR_INVALID_ARG, QNN_ERR_UNSUPPORTED, QNN_ERR_ALIGNMENT = -1, -2, -3
 QNN_ERR_WORKSPACE, QNN_ERR_CUDA, QNN_ERR_DEVICE_TIMEOUT = -4, -5, -6
 QNN_ENC_UNSIGNED, QNN_ENC_SIGNED, QNN_ENC_BIPOLAR = 0, 1, 2
-QNN_FMT_BITPLANES, QNN_FMT_INT8 = 0, 1
+QNN_FMT_BITPLANES, QNN_FMT_INT8, QNN_FMT_FIELDS = 0, 1, 2
 QNN_PATH_AUTO, QNN_PATH_BITSERIAL, QNN_PATH_TCGEN05_I8 = 0, 1, 2
 
 EXPORTS = (

@@ -22,12 +22,13 @@ int sm_count() {
 }
 
 static bool valid_fmt(int fmt) { return fmt == QNN_FMT_BITPLANES || fmt == QNN_FMT_INT8; }
+static int field_bits(int bits) { return bits == 1 ? 1 : (bits == 2 ? 2 : 4); }
 
 static qnn_status check_gemm_desc(const qnn_gemm_desc *d, bool has_thr, int *path_out) {
     if (!d) return QNN_ERR_INVALID_ARG;
     if (d->M <= 0 || d->N <= 0 || d->K <= 0) return QNN_ERR_INVALID_ARG;
     if (d->w_bits < 1 || d->w_bits > 8 || d->a_bits < 1 || d->a_bits > 8) return QNN_ERR_INVALID_ARG;
-    if (!valid_fmt(d->w_fmt) || !valid_fmt(d->a_fmt)) return QNN_ERR_INVALID_ARG;
+    if (!(valid_fmt(d->w_fmt) || d->w_fmt == QNN_FMT_FIELDS) || !valid_fmt(d->a_fmt)) return QNN_ERR_INVALID_ARG;
     if (d->w_enc < 0 || d->w_enc > 2 || d->a_enc < 0 || d->a_enc > 2) return QNN_ERR_INVALID_ARG;
     if (d->path < QNN_PATH_AUTO || d->path > QNN_PATH_TCGEN05_I8) return QNN_ERR_INVALID_ARG;
     if (has_thr) {
@@ -35,6 +36,13 @@ static qnn_status check_gemm_desc(const qnn_gemm_desc *d, bool has_thr, int *pat
         if (!valid_fmt(d->out_fmt)) return QNN_ERR_INVALID_ARG;
     }
     if (!valid_enc(d->w_enc, d->w_bits) || !valid_enc(d->a_enc, d->a_bits)) return QNN_ERR_UNSUPPORTED;
+    if (d->w_fmt == QNN_FMT_FIELDS) {
+        // packed w-bit weights against 8-bit activation containers: the few-column kernel only
+        if (d->a_fmt != QNN_FMT_INT8 || d->path == QNN_PATH_BITSERIAL) return QNN_ERR_UNSUPPORTED;
+        if (!gemv_fields_fits(d, has_thr)) return QNN_ERR_UNSUPPORTED;
+        if (path_out) *path_out = QNN_PATH_TCGEN05_I8;
+        return QNN_OK;
+    }
     if (d->w_fmt != d->a_fmt) return QNN_ERR_UNSUPPORTED;
     int path = d->path;
     if (path == QNN_PATH_AUTO)
@@ -113,21 +121,24 @@ size_t qnn_packed_ld(int K, int fmt) {
     if (K <= 0) return 0;
     if (fmt == QNN_FMT_BITPLANES) return (size_t)ceil_div(K, 32);
     if (fmt == QNN_FMT_INT8) return (size_t)round_up(K, 16);
-    return 0;
+    return 0;           // QNN_FMT_FIELDS: the pitch depends on the bit width, see qnn_packed_bytes
 }
 
 size_t qnn_packed_bytes(const qnn_pack_desc *d) {
     if (!d || d->rows <= 0 || d->K <= 0 || d->bits < 1 || d->bits > 8) return 0;
     if (d->fmt == QNN_FMT_BITPLANES) return (size_t)d->bits * d->rows * qnn_packed_ld(d->K, d->fmt) * 4;
     if (d->fmt == QNN_FMT_INT8) return (size_t)d->rows * qnn_packed_ld(d->K, d->fmt);
+    if (d->fmt == QNN_FMT_FIELDS && d->bits <= 4)
+        return (size_t)d->rows * 32 * ceil_div(d->K, 32 * (8 / field_bits(d->bits)));
     return 0;
 }
 
 qnn_status qnn_pack(const qnn_pack_desc *d, const void *logical, void *packed, void *stream) {
     if (!d || !logical || !packed) return QNN_ERR_INVALID_ARG;
     if (d->rows <= 0 || d->K <= 0 || d->bits < 1 || d->bits > 8) return QNN_ERR_INVALID_ARG;
-    if (!valid_fmt(d->fmt) || d->enc < 0 || d->enc > 2) return QNN_ERR_INVALID_ARG;
+    if (!(valid_fmt(d->fmt) || d->fmt == QNN_FMT_FIELDS) || d->enc < 0 || d->enc > 2) return QNN_ERR_INVALID_ARG;
     if (!valid_enc(d->enc, d->bits)) return QNN_ERR_UNSUPPORTED;
+    if (d->fmt == QNN_FMT_FIELDS && d->bits > 4) return QNN_ERR_UNSUPPORTED;
     if (!aligned16(logical) || !aligned16(packed)) return QNN_ERR_ALIGNMENT;
     return pack_launch(d, logical, packed, (cudaStream_t)stream);
 }
@@ -154,6 +165,7 @@ qnn_status qnn_qgemm(const qnn_gemm_desc *d, const void *W, const void *A, const
     if (!W || !A || !out) return QNN_ERR_INVALID_ARG;
     if (!aligned16(W) || !aligned16(A) || !aligned16(out) || (thr && (reinterpret_cast<uintptr_t>(thr) & 3u)))
         return QNN_ERR_ALIGNMENT;
+    if (d->w_fmt == QNN_FMT_FIELDS) return gemv_fields_launch(d, W, A, thr, out, (cudaStream_t)stream);
     // 8-bit containers with a handful of columns and no path forced: byte dot products,
     // one warp per weight row (a tensor-core tile would be almost empty)
     if (d->path == QNN_PATH_AUTO && d->w_fmt == QNN_FMT_INT8 && gemv_i8_fits(d))

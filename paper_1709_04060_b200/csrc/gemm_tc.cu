@@ -1023,6 +1023,10 @@ static bool make_map(CUtensorMap *map, const void *base, int rows, int K, int ld
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+bool tc_make_tile_map(CUtensorMap *map, const void *base, int rows, int row_bytes, int ld, int box_rows) {
+    return make_map(map, base, rows, row_bytes, ld, box_rows);
+}
+
 typedef CUresult (*EncodeIm2colFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                    const cuuint64_t *, const int *, const int *, cuuint32_t, cuuint32_t,
                                    const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,

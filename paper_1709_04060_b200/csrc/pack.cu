@@ -121,8 +121,45 @@ __global__ void pack_int8_kernel(const uint8_t *__restrict__ logical, uint8_t *_
     *reinterpret_cast<uint4 *>(packed + (size_t)r * ld + c * 16) = make_uint4(o[0], o[1], o[2], o[3]);
 }
 
+// QNN_FMT_FIELDS: one thread per packed 32-bit word.  Byte j of 32-byte group g of a row holds,
+// at bit position f*s, the field of element 32*S*g + 32*s + j (S = 8/f fields per byte).
+__global__ void pack_fields_kernel(const uint8_t *__restrict__ logical, uint32_t *__restrict__ packed,
+                                   int rows, int K, int ldw, int bits, int enc, int f) {
+    const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    if (idx >= (long long)rows * ldw) return;
+    const int r = (int)(idx / ldw);
+    const int w = (int)(idx - (long long)r * ldw);
+    const int S = 8 / f;
+    const int g = w >> 3, j0 = (w & 7) * 4;
+    const uint8_t *src = logical + (size_t)r * K;
+    uint32_t word = 0;
+    for (int b = 0; b < 4; ++b)
+        for (int s = 0; s < S; ++s) {
+            const long long k = (long long)32 * S * g + 32 * s + j0 + b;
+            if (k >= K) continue;
+            const int raw = (int8_t)src[k];
+            uint32_t u;
+            if (enc == QNN_ENC_BIPOLAR) u = raw > 0 ? 1u : 0u;
+            else if (enc == QNN_ENC_SIGNED) {
+                const int sh = 32 - bits;
+                u = (uint32_t)(((int32_t)((uint32_t)raw << sh) >> sh) + (1 << (bits - 1)));   // value - minimum
+            } else u = (uint32_t)raw & ((1u << bits) - 1u);
+            word |= u << (8 * b + f * s);
+        }
+    packed[idx] = word;
+}
+
 qnn_status pack_launch(const qnn_pack_desc *d, const void *logical, void *packed, cudaStream_t s) {
     const int threads = 256;
+    if (d->fmt == QNN_FMT_FIELDS) {
+        const int f = d->bits == 1 ? 1 : (d->bits == 2 ? 2 : 4);
+        const int ldw = 8 * ceil_div(d->K, 32 * (8 / f));           // words per packed row
+        const long long total = (long long)d->rows * ldw;
+        pack_fields_kernel<<<(unsigned)((total + threads - 1) / threads), threads, 0, s>>>(
+            (const uint8_t *)logical, (uint32_t *)packed, d->rows, d->K, ldw, d->bits, d->enc, f);
+        count_launch();
+        return launch_status();
+    }
     if (d->fmt == QNN_FMT_BITPLANES) {
         const int kw = ceil_div(d->K, 32);
         const long long total = (long long)d->rows * kw;

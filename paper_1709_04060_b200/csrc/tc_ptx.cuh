@@ -169,6 +169,11 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar_cluster_addr) {
                  ::"r"(bar_cluster_addr) : "memory");
 }
 
+// Tensor map over a byte matrix [rows][row_bytes] at pitch ld (a multiple of 16): boxes of 128
+// bytes x box_rows rows, written to shared memory with the 128-byte swizzle; out-of-range bytes
+// and rows read as zeros.  Host side.
+bool tc_make_tile_map(CUtensorMap *map, const void *base, int rows, int row_bytes, int ld, int box_rows);
+
 // Address of the library's device status word on the current device (host side; null on a
 // CUDA error).  Kernels outside the translation unit that defines the word get it as an argument.
 int *device_status_word();

@@ -35,7 +35,28 @@ def unpack_int8(buf: np.ndarray, rows: int, K: int, enc: int) -> np.ndarray:
     return (m if enc == UNSIGNED else m.view(np.int8)).astype(np.int32)
 
 
+def unpack_fields(buf: np.ndarray, bits: int, rows: int, K: int, enc: int) -> np.ndarray:
+    """QNN_FMT_FIELDS [rows][ldf] bytes -> logical int32 [rows][K]; also checks zero pad fields.
+    Element k sits in byte 32 g + j at bit f s, g = k // (32 S), s = (k % (32 S)) // 32, j = k % 32."""
+    f = 1 if bits == 1 else (2 if bits == 2 else 4)
+    S = 8 // f
+    groups = (K + 32 * S - 1) // (32 * S)
+    ldf = 32 * groups
+    m = buf.view(np.uint8)[: rows * ldf].reshape(rows, groups, 32).astype(np.int32)
+    fields = np.stack([(m >> (f * s)) & ((1 << f) - 1) for s in range(S)], axis=2)     # [rows][g][s][j]
+    u = fields.reshape(rows, groups * 32 * S)
+    assert not u[:, K:].any(), "pad fields must be zero"
+    u = u[:, :K]
+    if enc == BIPOLAR:
+        return 2 * u - 1
+    if enc == SIGNED:
+        return u - (1 << (bits - 1))
+    return u
+
+
 def unpack_operand(buf, fmt, bits, rows, K, enc):
+    if fmt == 2:
+        return unpack_fields(buf, bits, rows, K, enc)
     return unpack_planes(buf, bits, rows, K, enc) if fmt == 0 else unpack_int8(buf, rows, K, enc)
 
 
