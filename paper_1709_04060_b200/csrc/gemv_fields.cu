@@ -21,18 +21,21 @@
 // depth indices: the activation operand is the plain [N][K] byte matrix, untouched.
 // Fields hold the value minus the encoding's minimum (u = v - vmin >= 0), or the bit of a
 // bipolar weight (v = 2u - 1): sum_k v_k a_k = scale * sum_k u_k a_k + offset * sum_k a_k,
-// and the column sums of the activations are formed once per CTA from shared memory.
+// and the column sums of the activations come out of the same MMAs: the first tensor-memory lane
+// past the block's rows holds a row of ones.
 //
 // CTA = one block of up to 128 weight rows x one slice of the depth; the CTAs of a cluster
 // split the depth of the same rows and hand their int32 partial sums to the cluster's first
 // CTA through distributed shared memory before the thresholds are counted.  Warp roles:
-//   warp 0     producer: TMA loads of the activation k-blocks (16 rows x 128 bytes each) and of
-//              the packed weight stages (rows x 128 bytes, 128-byte swizzle) into a ring
-//   warp 1     allocates tensor memory; one lane issues the MMAs (128 x 16 x 32 per instruction,
-//              row operand from tensor memory, activations from shared memory)
-//   warps 2-9  expansion, two groups of four warps (one warp per lane quarter), each group
-//              filling one of two operand buffers in tensor memory in turn; group 0 then runs
-//              the epilogue, group 1 forms the activation column sums
+//   warp 0       producer: TMA loads of the packed weight stages (rows x 128 bytes, 128-byte
+//                swizzle) into a ring
+//   warp 1       allocates tensor memory; one lane issues the MMAs (128 x 16 x 32 per
+//                instruction, row operand from tensor memory, activations from shared memory)
+//   warps 2-9    expansion, two groups of four warps (one warp per lane quarter) that take the
+//                chunks in turn and fill the three operand buffers in tensor memory round
+//                robin; group 0 then runs the epilogue
+//   warp 10      TMA loads of the slice's activation k-blocks (16 rows x 128 bytes each, all
+//                resident)
 // Every wait is bounded; on expiry the CTA records QNN_ERR_DEVICE_TIMEOUT and drains.
 #include <cuda.h>
 
@@ -48,9 +51,10 @@ constexpr int GF_MAX_ST = 32;               // stages per depth slice (one barri
 constexpr int GF_ACT_KB_BYTES = GF_NPAD * 128;       // one activation k-block in shared memory
 constexpr int GF_ACT_MAX_BYTES = 100 * 1024;
 constexpr int GF_MAX_SPLIT = 4;
-constexpr int GF_THREADS = 32 * 10;
+constexpr int GF_THREADS = 32 * 11;
+constexpr int GF_NB = 3;                    // operand buffers in tensor memory (128 columns apart)
 constexpr uint32_t GF_TMEM_COLS = 512;
-constexpr uint32_t GF_ACC_COL = 256;        // accumulators at columns 256.., operand buffers at 0 and 128
+constexpr uint32_t GF_ACC_COL = 128 * GF_NB;         // accumulators behind the operand buffers
 
 enum { GF_OUT_RAW = 0, GF_OUT_U8 = 1, GF_OUT_PLANES = 2 };
 
@@ -71,11 +75,10 @@ struct GfParams {
 struct GfBars {
     alignas(8) uint64_t full[GF_NS];
     uint64_t empty[GF_NS];
-    uint64_t a_full[2];
-    uint64_t a_empty[2];
+    uint64_t a_full[GF_NB];
+    uint64_t a_empty[GF_NB];
     uint64_t act_full[GF_MAX_ST];
     uint64_t acc_full;
-    uint64_t colsum_done;
     int colsum[GF_NPAD];
     uint32_t tmem_base;
     int abort_flag;
@@ -106,11 +109,11 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t *r) {
           "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]) : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int (&r)[16]) {
+__device__ __forceinline__ void tmem_ld_fence() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, int (&r)[16]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n\t"
-        "tcgen05.wait::ld.sync.aligned;"
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr) : "memory");
@@ -133,8 +136,8 @@ __global__ void __launch_bounds__(GF_THREADS, 1)
 gemv_fields_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_act,
                    const GfParams p) {
     constexpr int S = 8 / F;                       // fields per byte = accumulators
-    constexpr int CG = F == 1 ? 2 : 4;             // 32-byte groups per operand buffer fill ("chunk")
-    constexpr int CPS = 4 / CG;                    // chunks per stage
+    constexpr int CG = 16 / S;                     // 32-byte groups per operand buffer fill ("chunk"): 128 columns
+    constexpr int GPS = 4;                         // groups per stage (128 packed bytes per row)
     constexpr uint32_t FMASK = F == 1 ? 0x01010101u : (F == 2 ? 0x03030303u : 0x0F0F0F0Fu);
     extern __shared__ uint8_t gf_raw[];
     uint8_t *base = gf_raw + ((1024u - (smem_u32(gf_raw) & 1023u)) & 1023u);
@@ -144,8 +147,12 @@ gemv_fields_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
     const int m0 = block * p.R;
     const int st0 = (int)rank * p.st_per;
     const int nst_local = min(p.nst, st0 + p.st_per) - st0;          // >= 1 by construction
-    const int nkb = nst_local * S;                                   // activation k-blocks of this slice
+    const int nchunks = (nst_local * GPS + CG - 1) / CG;
     const uint32_t stage_bytes = (uint32_t)p.R * GF_STAGE_ROW_BYTES;
+    // The blocks walk the stages of their slice in rotated orders (integer sums do not care): all
+    // blocks read the same activation bytes, and in lock step they would all ask for the same
+    // lines of L2 at the same time.
+    const int rot = block % nst_local;
 
     uint8_t *ring = base;                                                       // [GF_NS][128 rows x 128 B]
     uint8_t *act = ring + GF_NS * 128 * GF_STAGE_ROW_BYTES;                     // [st_per * S][16 x 128 B]
@@ -155,11 +162,11 @@ gemv_fields_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
     volatile int *abort_flag = &bar.abort_flag;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < GF_NS; ++s) { mbar_init(&bar.full[s], 1); mbar_init(&bar.empty[s], 4 * CPS); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&bar.a_full[b], 4); mbar_init(&bar.a_empty[b], 1); }
+        // a stage is read by the four warps of every group that has a chunk (or part of one) in it
+        for (int s = 0; s < GF_NS; ++s) { mbar_init(&bar.full[s], 1); mbar_init(&bar.empty[s], CG < GPS ? 8 : 4); }
+        for (int b = 0; b < GF_NB; ++b) { mbar_init(&bar.a_full[b], 4); mbar_init(&bar.a_empty[b], 1); }
         for (int j = 0; j < GF_MAX_ST; ++j) mbar_init(&bar.act_full[j], 1);
         mbar_init(&bar.acc_full, 1);
-        mbar_init(&bar.colsum_done, 4);
         bar.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -172,7 +179,7 @@ gemv_fields_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
     const uint32_t tmem_base = bar.tmem_base;
 
     // state the row-owning threads (expansion group 0) carry from the main loop into the epilogue
-    const int h = warp >= 2 ? (warp - 2) >> 2 : -1, q = warp & 3;
+    const int h = (warp >= 2 && warp < 10) ? (warp - 2) >> 2 : -1, q = warp & 3;
     const int r = q * 32 + lane;                                     // weight row of this thread = lane of tensor memory
     const int m = m0 + r;
     const int n_thr = p.out_mode == GF_OUT_RAW ? 0 : (1 << p.out_bits) - 1;
@@ -181,138 +188,176 @@ gemv_fields_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
     for (int n = 0; n < GF_NPAD; ++n) acc[n] = 0;
 
     if (warp == 0) {
-        // ---------------------------------------------------------------- producer
+        // ------------------------------------------------- producer of the packed weight stages
         if (lane == 0) {
-            bool ok = true;
-            for (int j = 0; ok && j < nst_local; ++j) {
-                // the activation k-blocks that stage j's elements meet, then the packed weights
-                mbar_arrive_expect_tx(&bar.act_full[j], (uint32_t)S * GF_ACT_KB_BYTES);
-                for (int s = 0; s < S; ++s)
-                    tma_load_2d(act + (size_t)(j * S + s) * GF_ACT_KB_BYTES, &map_act, &bar.act_full[j],
-                                ((st0 + j) * S + s) * 128, 0);
+            for (int j = 0; j < nst_local; ++j) {
                 const int slot = j % GF_NS;
-                if (!(ok = mbar_wait(&bar.empty[slot], ((j / GF_NS) & 1) ^ 1, abort_flag, p.status))) break;
+                if (!mbar_wait(&bar.empty[slot], ((j / GF_NS) & 1) ^ 1, abort_flag, p.status)) break;
                 mbar_arrive_expect_tx(&bar.full[slot], stage_bytes);
                 tma_load_2d(ring + (size_t)slot * 128 * GF_STAGE_ROW_BYTES, &map_w, &bar.full[slot],
-                            (st0 + j) * GF_STAGE_ROW_BYTES, m0);
-            }
-            if (!ok) {
-                // gave up: let the copies already issued land before the CTA exits
-                for (int j = 0; j < nst_local; ++j)
-                    if (!mbar_wait(&bar.act_full[j], 0, abort_flag, p.status)) break;
+                            (st0 + (j + rot) % nst_local) * GF_STAGE_ROW_BYTES, m0);
             }
         }
         __syncwarp();
     } else if (warp == 1) {
         // -------------------------------------------------------------- MMA issuer
+        // A 128 x 16 x 32 MMA keeps the tensor pipe busy for 64 cycles only and the pipe's queue is
+        // short, so whatever this thread does between two MMAs (a barrier poll costs about 150
+        // cycles while the pipe reads shared memory) shows up as idle pipe: one poll per chunk,
+        // placed where half of the chunk's MMAs are queued, and no other work in the loop.
         if (lane == 0) {
+            // act_ok: stages whose activation k-blocks are known to have landed
             bool ok = true;
-            const int nchunks = nst_local * CPS;
+            int act_ok = 0;
+            const int first_stages = min(nst_local, (CG + GPS - 1) / GPS);
+            for (; ok && act_ok < first_stages; ++act_ok) ok = mbar_wait_spin(&bar.act_full[act_ok], 0, abort_flag, p.status);
+            if (ok) ok = mbar_wait_spin(&bar.a_full[0], 0, abort_flag, p.status);
+            tc_fence_after();
+            uint64_t db_chunk = umma_smem_desc(smem_u32(act));       // first activation slice of the chunk
+            uint32_t buf = 0, use = 0;                               // operand buffer of the chunk, its use count
             for (int c = 0; ok && c < nchunks; ++c) {
-                const int j = c / CPS, part = c % CPS;
-                const uint32_t buf = c & 1;
-                if (part == 0 && !(ok = mbar_wait(&bar.act_full[j], 0, abort_flag, p.status))) break;
-                if (!(ok = mbar_wait(&bar.a_full[buf], (c >> 1) & 1, abort_flag, p.status))) break;
-                tc_fence_after();
+                const uint32_t a_tmem = tmem_base + buf * 128u;
+                uint32_t nbuf = buf + 1, nuse = use;
+                if (nbuf == GF_NB) { nbuf = 0; ++nuse; }
+                // a chunk is MPC MMAs unless the slice ends inside it
+                const int groups = min(CG, 4 * nst_local - c * CG);
 #pragma unroll
                 for (int gl = 0; gl < CG; ++gl) {
-                    const int g = part * CG + gl;                    // 32-byte group within the stage
+                    if (gl < groups) {
 #pragma unroll
-                    for (int s = 0; s < S; ++s) {
-                        const int slice = S * (4 * j + g) + s;       // 32-byte slice of the activation rows
-                        const uint64_t db = umma_smem_desc(smem_u32(act + (size_t)(slice >> 2) * GF_ACT_KB_BYTES)) +
-                                            2 * (slice & 3);
-                        umma_i8_a_tmem(tmem_base + GF_ACC_COL + (uint32_t)(s * GF_NPAD),
-                                       tmem_base + buf * 128u + (uint32_t)((gl * S + s) * 8), db, p.idesc,
-                                       (j | g) != 0);
+                        for (int s = 0; s < S; ++s) {
+                            const int rel = gl * S + s;              // slice within the chunk (compile time)
+                            umma_i8_a_tmem(tmem_base + GF_ACC_COL + (uint32_t)(s * GF_NPAD), a_tmem + (uint32_t)(rel * 8),
+                                           db_chunk + (uint64_t)((rel >> 2) * 128 + (rel & 3) * 2), p.idesc,
+                                           (c | gl) != 0);
+                        }
+                    }
+                    if (gl == CG / 2 - 1 && c + 1 < nchunks) {
+                        // the next chunk never depends on this one's completion
+                        const int need = min(nst_local, ((c + 2) * CG + GPS - 1) / GPS);     // stages up to its end
+                        for (; ok && act_ok < need; ++act_ok) ok = mbar_wait_spin(&bar.act_full[act_ok], 0, abort_flag, p.status);
+                        if (ok) ok = mbar_wait_spin(&bar.a_full[nbuf], nuse & 1u, abort_flag, p.status);
+                        tc_fence_after();
+                        if (!ok) break;
                     }
                 }
+                if (!ok) break;
                 umma_commit(&bar.a_empty[buf]);
+                db_chunk += (uint64_t)(S * CG / 4) * 128u;           // S * CG slices = S * CG / 4 k-blocks
+                buf = nbuf; use = nuse;
             }
             if (ok) umma_commit(&bar.acc_full);
         }
         __syncwarp();
+    } else if (warp == 10) {
+        // -------------------------- activations: all k-blocks of the slice stay resident
+        if (lane == 0) {
+            for (int j = 0; j < nst_local; ++j) {
+                mbar_arrive_expect_tx(&bar.act_full[j], (uint32_t)S * GF_ACT_KB_BYTES);
+                for (int s = 0; s < S; ++s)
+                    tma_load_2d(act + (size_t)(j * S + s) * GF_ACT_KB_BYTES, &map_act, &bar.act_full[j],
+                                ((st0 + (j + rot) % nst_local) * S + s) * 128, 0);
+            }
+        }
+        __syncwarp();
     } else {
-        // ------------------------------------------------ expansion, then epilogue / column sums
+        // -------------------------------------------------------- expansion, then epilogue
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-        const int nchunks = nst_local * CPS;
+        if (h == 0) {
+            // thresholds of this thread's row: in registers long before they are needed
+#pragma unroll
+            for (int i = 0; i < 15; ++i)
+                t[i] = (i < n_thr && m < p.M && r < p.R) ? __ldg(p.thr + (size_t)m * n_thr + i) : 0x7fffffff;
+        }
+        // Lane R of tensor memory (the first one past the block's rows) carries a row of ones: its
+        // accumulators collect sum_k a[n][k], the column sums that the weight encoding's offset
+        // multiplies, at no extra cost.
+        const bool ones_row = r == p.R;
+        const uint32_t fill = ones_row ? 0xFFFFFFFFu : 0u;           // ones row: every field mask sees all bits ...
+        uint32_t fmask[S];
+#pragma unroll
+        for (int s = 0; s < S; ++s) fmask[s] = ones_row ? 0x01010101u : (FMASK << (F * s));    // ... and keeps a 1
         bool ok = true;
         for (int c = h; c < nchunks; c += 2) {
-            const int j = c / CPS, part = c % CPS, slot = j % GF_NS;
-            if (!(ok = gf_warp_wait(&bar.full[slot], (j / GF_NS) & 1, lane, abort_flag, p.status))) break;
-            if (!(ok = gf_warp_wait(&bar.a_empty[h], ((c >> 1) & 1) ^ 1, lane, abort_flag, p.status))) break;
+            const int buf = c % GF_NB;
+            const int g_first = c * CG;                              // first 32-byte group of the chunk (slice-relative)
+            const int groups = min(CG, GPS * nst_local - g_first);
+            const int j_first = g_first / GPS, j_last = (g_first + groups - 1) / GPS;
+            if (lane == 0) {
+                ok = mbar_wait_spin(&bar.a_empty[buf], (uint32_t)(((c / GF_NB) & 1) ^ 1), abort_flag, p.status);
+                for (int j = j_first; ok && j <= j_last; ++j)
+                    ok = mbar_wait_spin(&bar.full[j % GF_NS], (j / GF_NS) & 1, abort_flag, p.status);
+            }
+            ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+            if (!ok) break;
             tc_fence_after();
-            const uint32_t row = smem_u32(ring + (size_t)slot * 128 * GF_STAGE_ROW_BYTES) + (uint32_t)r * 128u;
 #pragma unroll
             for (int gl = 0; gl < CG; ++gl) {
-                const int g = part * CG + gl;
-                const uint4 lo = lds128(row + (uint32_t)(((2 * g) ^ (r & 7)) << 4));
-                const uint4 hi = lds128(row + (uint32_t)(((2 * g + 1) ^ (r & 7)) << 4));
-                const uint32_t x[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
-                uint32_t y[8 * S];
+                if (gl < groups) {
+                    const int gg = g_first + gl, j = gg / GPS, g = gg % GPS;
+                    const uint32_t row = smem_u32(ring + (size_t)(j % GF_NS) * 128 * GF_STAGE_ROW_BYTES) + (uint32_t)r * 128u;
+                    const uint4 lo = lds128(row + (uint32_t)(((2 * g) ^ (r & 7)) << 4));
+                    const uint4 hi = lds128(row + (uint32_t)(((2 * g + 1) ^ (r & 7)) << 4));
+                    const uint32_t x[8] = {lo.x | fill, lo.y | fill, lo.z | fill, lo.w | fill,
+                                           hi.x | fill, hi.y | fill, hi.z | fill, hi.w | fill};
+                    uint32_t y[8 * S];
 #pragma unroll
-                for (int s = 0; s < S; ++s)
+                    for (int s = 0; s < S; ++s)
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) y[8 * s + i] = x[i] & (FMASK << (F * s));
-                const uint32_t taddr = tmem_base + lane_addr + (uint32_t)h * 128u + (uint32_t)(gl * S * 8);
-                if (S == 2) {
-                    tmem_st16(taddr, y);
-                } else {
+                        for (int i = 0; i < 8; ++i) y[8 * s + i] = x[i] & fmask[s];
+                    const uint32_t taddr = tmem_base + lane_addr + (uint32_t)buf * 128u + (uint32_t)(gl * S * 8);
+                    if (S == 2) {
+                        tmem_st16(taddr, y);
+                    } else {
 #pragma unroll
-                    for (int v = 0; v < S / 4; ++v) tmem_st32(taddr + 32u * v, y + 32 * v);
+                        for (int v = 0; v < S / 4; ++v) tmem_st32(taddr + 32u * v, y + 32 * v);
+                    }
                 }
             }
             tmem_st_wait();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(&bar.empty[slot]);       // this warp has read its part of the stage (its only visit)
-                mbar_arrive(&bar.a_full[h]);
+                mbar_arrive(&bar.a_full[buf]);
+                // this warp has read its part of these stages (its only visit to them)
+                for (int j = j_first; j <= j_last; ++j) mbar_arrive(&bar.empty[j % GF_NS]);
             }
         }
 
-        if (h == 1) {
-            // column sums of this slice's activations (only where the weight encoding has an offset)
-            if (ok && p.w_off != 0) {
-                const int tix = threadIdx.x - 32 * 6;                // 0..127
-                const int n = tix & 15, part = tix >> 4;
-                for (int j = 0; ok && j < nst_local; ++j) ok = mbar_wait(&bar.act_full[j], 0, abort_flag, p.status);
-                int sum = 0;
-                if (ok) {
-                    for (int kb = part; kb < nkb; kb += 8) {
-                        const uint32_t a = smem_u32(act + (size_t)kb * GF_ACT_KB_BYTES) + (uint32_t)n * 128u;
-#pragma unroll
-                        for (int v = 0; v < 8; ++v) {
-                            const uint4 d = lds128(a + 16u * v);
-                            if (p.a_signed)
-                                sum = __dp4a((int)d.x, 0x01010101, __dp4a((int)d.y, 0x01010101,
-                                      __dp4a((int)d.z, 0x01010101, __dp4a((int)d.w, 0x01010101, sum))));
-                            else
-                                sum = (int)__dp4a(d.x, 0x01010101u, __dp4a(d.y, 0x01010101u,
-                                      __dp4a(d.z, 0x01010101u, __dp4a(d.w, 0x01010101u, (unsigned)sum))));
-                        }
-                    }
-                    if (sum != 0) atomicAdd(&bar.colsum[n], sum);
-                }
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bar.colsum_done);
-        } else {
-            // thresholds of this thread's row, loaded while the last MMAs run
-#pragma unroll
-            for (int i = 0; i < 15; ++i)
-                t[i] = (i < n_thr && m < p.M && r < p.R) ? __ldg(p.thr + (size_t)m * n_thr + i) : 0x7fffffff;
-            if (ok) ok = gf_warp_wait(&bar.acc_full, 0, lane, abort_flag, p.status);
-            if (ok && p.w_off != 0) ok = gf_warp_wait(&bar.colsum_done, 0, lane, abort_flag, p.status);
+        if (h == 0) {
+            if (lane == 0 && ok) ok = mbar_wait_spin(&bar.acc_full, 0, abort_flag, p.status);
+            ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
             if (ok) {
                 tc_fence_after();
+                // the S accumulators of this row, four at a time
+                int ones[GF_NPAD];
 #pragma unroll
-                for (int s = 0; s < S; ++s) {
-                    int d[GF_NPAD];
-                    tmem_ld16(tmem_base + lane_addr + GF_ACC_COL + (uint32_t)(s * GF_NPAD), d);
+                for (int n = 0; n < GF_NPAD; ++n) ones[n] = 0;
 #pragma unroll
-                    for (int n = 0; n < GF_NPAD; ++n) acc[n] += d[n] >> (F * s);     // exact: a multiple of 2^(F s)
+                for (int s0 = 0; s0 < S; s0 += 4) {
+                    int d[4][GF_NPAD];
+#pragma unroll
+                    for (int s = 0; s < 4; ++s)
+                        if (s0 + s < S) tmem_ld16_issue(tmem_base + lane_addr + GF_ACC_COL + (uint32_t)((s0 + s) * GF_NPAD), d[s]);
+                    tmem_ld_fence();
+#pragma unroll
+                    for (int s = 0; s < 4; ++s)
+                        if (s0 + s < S) {
+#pragma unroll
+                            for (int n = 0; n < GF_NPAD; ++n) {
+                                acc[n] += d[s][n] >> (F * (s0 + s));     // exact: a multiple of 2^(F s)
+                                ones[n] += d[s][n];                      // the row of ones is not scaled
+                            }
+                        }
                 }
+                if (ones_row) {
+#pragma unroll
+                    for (int n = 0; n < GF_NPAD; ++n) bar.colsum[n] = ones[n];
+                }
+            }
+            // the four epilogue warps meet: the column sums are in shared memory
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (ok) {
 #pragma unroll
                 for (int n = 0; n < GF_NPAD; ++n) acc[n] = p.w_scale * acc[n] + p.w_off * bar.colsum[n];
                 if (rank != 0) {
@@ -345,39 +390,35 @@ gemv_fields_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
             }
         }
         const bool row_ok = r < p.R && m < p.M;
-        if (p.out_mode == GF_OUT_RAW) {
-            if (row_ok) {
+        const int mw = (p.M + 31) >> 5, word = (m0 >> 5) + q;
 #pragma unroll
-                for (int n = 0; n < GF_NPAD; ++n)
-                    if (n < p.N) reinterpret_cast<int32_t *>(p.out)[(size_t)n * p.M + m] = acc[n];
+        for (int n = 0; n < GF_NPAD; ++n) {
+            if (n >= p.N) break;                                     // uniform
+            if (p.out_mode == GF_OUT_RAW) {
+                if (row_ok) reinterpret_cast<int32_t *>(p.out)[(size_t)n * p.M + m] = acc[n];
+                continue;
             }
-        } else {
-            int code[GF_NPAD];
+            // T(x, t): thresholds past the row's count hold INT32_MAX and are not looked at
+            const int x = acc[n];
+            int code = (x >= t[0]) ? 1 : 0;
+            if (p.out_bits >= 2) code += ((x >= t[1]) ? 1 : 0) + ((x >= t[2]) ? 1 : 0);
+            if (p.out_bits >= 3) code += ((x >= t[3]) ? 1 : 0) + ((x >= t[4]) ? 1 : 0) + ((x >= t[5]) ? 1 : 0) + ((x >= t[6]) ? 1 : 0);
+            if (p.out_bits >= 4) {
+                int c2 = 0;
 #pragma unroll
-            for (int n = 0; n < GF_NPAD; ++n) {
-                int cnt = 0;
-#pragma unroll
-                for (int i = 0; i < 15; ++i) cnt += (i < n_thr && acc[n] >= t[i]) ? 1 : 0;
-                code[n] = row_ok ? cnt : 0;
+                for (int i = 7; i < 15; ++i) c2 += (x >= t[i]) ? 1 : 0;
+                code += c2;
             }
+            if (!row_ok) code = 0;
             if (p.out_mode == GF_OUT_U8) {
-                if (r < p.R && m < p.ld_out) {                   // pad bytes of a row are written as zeros
-#pragma unroll
-                    for (int n = 0; n < GF_NPAD; ++n)
-                        if (n < p.N) reinterpret_cast<uint8_t *>(p.out)[(size_t)n * p.ld_out + m] = (uint8_t)code[n];
-                }
+                // pad bytes of an output row (m in [M, ld_out)) are written as zeros
+                if (r < p.R && m < p.ld_out) reinterpret_cast<uint8_t *>(p.out)[(size_t)n * p.ld_out + m] = (uint8_t)code;
             } else {
                 // 32 rows of a warp are one word of the channel-interleaved layout (R is a multiple of 32)
-                const int mw = (p.M + 31) >> 5, word = (m0 >> 5) + q;
-#pragma unroll
-                for (int n = 0; n < GF_NPAD; ++n) {
-                    if (n < p.N) {
-                        for (int b = 0; b < p.out_bits; ++b) {
-                            const uint32_t bits = __ballot_sync(0xffffffffu, (code[n] >> b) & 1);
-                            if (lane == 0 && q * 32 < p.R && word < mw)
-                                reinterpret_cast<uint32_t *>(p.out)[((size_t)b * p.N + n) * mw + word] = bits;
-                        }
-                    }
+                for (int b = 0; b < p.out_bits; ++b) {
+                    const uint32_t bits = __ballot_sync(0xffffffffu, (code >> b) & 1);
+                    if (lane == 0 && q * 32 < p.R && word < mw)
+                        reinterpret_cast<uint32_t *>(p.out)[((size_t)b * p.N + n) * mw + word] = bits;
                 }
             }
         }
@@ -411,7 +452,7 @@ static bool gf_plan(const qnn_gemm_desc *d, bool has_thr, GfPlan *pl) {
         if (st_per > GF_MAX_ST || (size_t)st_per * pl->S * GF_ACT_KB_BYTES > (size_t)GF_ACT_MAX_BYTES) continue;
         const int target = sms / sk > 0 ? sms / sk : 1;
         int R = round_up(ceil_div(cover, target), gran);
-        if (R > 128) R = 128;
+        if (R > 128 - gran) R = 128 - gran;                                // one lane is left for the row of ones
         const int nblocks = ceil_div(cover, R);
         const long long ctas = (long long)nblocks * sk;
         const double waves = (double)((ctas + sms - 1) / sms);
@@ -467,10 +508,19 @@ qnn_status gemv_fields_launch(const qnn_gemm_desc *d, const void *W, const void 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(pl.nblocks * pl.sk)); cfg.blockDim = dim3(GF_THREADS);
     cfg.dynamicSmemBytes = smem; cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)pl.sk; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr; cfg.numAttrs = pl.sk > 1 ? 1 : 0;
+    cudaLaunchAttribute attr[2];
+    int na = 0;
+    // programmatic dependent launch: the CTAs set up (barriers, tensor memory) as SMs fall idle at
+    // the end of the previous kernel and wait in griddepcontrol.wait before touching global memory
+    attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+    if (pl.sk > 1) {
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = (unsigned)pl.sk; attr[na].val.clusterDim.y = 1; attr[na].val.clusterDim.z = 1;
+        ++na;
+    }
+    cfg.attrs = attr; cfg.numAttrs = na;
     cudaError_t e;
     if (pl.F == 1) e = cudaLaunchKernelEx(&cfg, gemv_fields_kernel<1>, mw, ma, p);
     else if (pl.F == 2) e = cudaLaunchKernelEx(&cfg, gemv_fields_kernel<2>, mw, ma, p);
