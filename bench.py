@@ -782,45 +782,62 @@ def run_extras(args):
 
 
 def run_shapes(args):
-    """Size sweep of Section 4.1.2 of the paper: every (rows, depth, cols) in {2^6 .. 2^12}^3 for
-    W1A1 (bipolar x bipolar) GEMM+threshold, on 8-bit containers (tensor cores, or byte dot
-    products below 9 columns) and on bit planes (bit-serial kernels), each timed by replaying a
-    CUDA graph of repeated calls.  Prints one JSON line with the per-shape times and the faster
-    operand format."""
+    """Size sweep of Section 4.1.2 of the paper: every (rows, depth, cols) in {2^6 .. 2^12}^3, for
+    every (w, a) in {1..4}^2 (--pairs restricts them; weights bipolar when w = 1, else signed;
+    activations unsigned), GEMM+threshold on 8-bit containers (tensor cores) and on bit planes
+    (bit-serial kernels), each timed by replaying a CUDA graph of repeated calls.  Prints one JSON
+    line per (w, a) with the per-shape times, the faster operand format and the kernel the library
+    chose, and a summary line."""
     import torch
     import __graft_entry__ as ge
     ge.build()
     from paper_1709_04060_b200 import binding as qb
     torch.cuda.set_device(0)
-    PL, I8, BIP = qb.QNN_FMT_BITPLANES, qb.QNN_FMT_INT8, qb.QNN_ENC_BIPOLAR
+    PL, I8 = qb.QNN_FMT_BITPLANES, qb.QNN_FMT_INT8
     dims = [2 ** e for e in range(6, 13)]
     if QUICK:
         dims = [64, 1024, 4096]
     g = torch.Generator(device="cuda").manual_seed(170904060)
-    big = (2 * torch.randint(0, 2, (4096, 4096), dtype=torch.int8, device="cuda", generator=g) - 1).contiguous()
-    thr_all = torch.randint(-32, 33, (4096, 1), dtype=torch.int32, device="cuda", generator=g)
-    rows = []
-    for M in dims:
-        for K in dims:
-            Wl = big[:M, :K].contiguous()
-            Wp = {f: qb.pack(Wl, 1, BIP, f) for f in (I8, PL)}
-            thr = thr_all[:M].contiguous()
-            for N in dims:
-                Al = big[4096 - N:, 4096 - K:].contiguous()
-                res = {"M": M, "K": K, "N": N}
-                for f, name in ((I8, "int8"), (PL, "bitplanes")):
-                    Ap = qb.pack(Al, 1, BIP, f)
-                    d = qb.gemm_desc(M, N, K, 1, 1, 1, BIP, BIP, f, I8)
-                    out = torch.empty(max(qb.qnn_gemm_out_bytes(d, True), 16), dtype=torch.uint8, device="cuda")
-                    reps = 10 if M * N * K < 2 ** 30 else 3
-                    ms = _time_calls(torch, lambda i: qb.check(qb.qnn_qgemm(d, Wp[f], Ap, thr, out)), reps, graph=True)
-                    res[name + "_us"] = round(1e3 * ms, 2)
-                res["gmacs_best"] = round(M * N * K / (min(res["int8_us"], res["bitplanes_us"]) * 1e-6) / 1e9, 1)
-                res["faster"] = "int8" if res["int8_us"] <= res["bitplanes_us"] else "bitplanes"
-                rows.append(res)
-    n_bit = sum(r["faster"] == "bitplanes" for r in rows)
-    print(json.dumps({"workload": "shapes", "precision": "W1A1 bipolar, 1 threshold per row", "shapes": len(rows),
-                      "bitplanes_faster": n_bit, "rows": rows}))
+    summary = []
+    for (w, a) in PAIRS:
+        w_enc = qb.QNN_ENC_BIPOLAR if w == 1 else qb.QNN_ENC_SIGNED
+        a_enc = qb.QNN_ENC_UNSIGNED
+        if w == 1:
+            bigW = (2 * torch.randint(0, 2, (4096, 4096), dtype=torch.int8, device="cuda", generator=g) - 1).contiguous()
+        else:
+            bigW = torch.randint(-(1 << (w - 1)), 1 << (w - 1), (4096, 4096), dtype=torch.int8, device="cuda", generator=g)
+        bigA = torch.randint(0, 1 << a, (4096, 4096), dtype=torch.uint8, device="cuda", generator=g)
+        n_thr = (1 << a) - 1
+        thr_all = torch.sort(torch.randint(-64, 65, (4096, n_thr), dtype=torch.int32, device="cuda", generator=g), dim=1).values.contiguous()
+        rows = []
+        for M in dims:
+            for K in dims:
+                Wl = bigW[:M, :K].contiguous()
+                Wp = {f: qb.pack(Wl, w, w_enc, f) for f in (I8, PL)}
+                thr = thr_all[:M].contiguous()
+                for N in dims:
+                    Al = bigA[4096 - N:, 4096 - K:].contiguous()
+                    res = {"M": M, "K": K, "N": N}
+                    for f, name in ((I8, "int8"), (PL, "bitplanes")):
+                        Ap = qb.pack(Al, a, a_enc, f)
+                        d = qb.gemm_desc(M, N, K, w, a, a, w_enc, a_enc, f, I8)
+                        out = torch.empty(max(qb.qnn_gemm_out_bytes(d, True), 16), dtype=torch.uint8, device="cuda")
+                        reps = 10 if M * N * K < 2 ** 30 else 3
+                        ms = _time_calls(torch, lambda i: qb.check(qb.qnn_qgemm(d, Wp[f], Ap, thr, out)), reps, graph=True)
+                        res[name + "_us"] = round(1e3 * ms, 2)
+                        res[name + "_kernel"] = qb.qnn_qgemm_kernel(d, True)
+                    res["gmacs_best"] = round(M * N * K / (min(res["int8_us"], res["bitplanes_us"]) * 1e-6) / 1e9, 1)
+                    res["faster"] = "int8" if res["int8_us"] <= res["bitplanes_us"] else "bitplanes"
+                    rows.append(res)
+        ratios = sorted(r["bitplanes_us"] / r["int8_us"] for r in rows)
+        line = {"workload": "shapes", "w": w, "a": a, "shapes": len(rows),
+                "bitplanes_faster": sum(r["faster"] == "bitplanes" for r in rows),
+                "ratio_bitplanes_over_int8": {"min": round(ratios[0], 2), "median": round(ratios[len(ratios) // 2], 2),
+                                              "max": round(ratios[-1], 2)},
+                "rows": rows}
+        print(json.dumps(line), flush=True)
+        summary.append({k: line[k] for k in ("w", "a", "shapes", "bitplanes_faster", "ratio_bitplanes_over_int8")})
+    print(json.dumps({"workload": "shapes_summary", "summary": summary}))
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one 4096^3 W1A2 launch of the (CTA-pair)

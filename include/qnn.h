@@ -149,6 +149,24 @@ qnn_status qnn_qgemm(const qnn_gemm_desc *d, const void *W, const void *A,
                      const int32_t *thr, void *out,
                      void *workspace, size_t workspace_bytes, void *stream);
 
+/* Which kernel qnn_qgemm runs for this problem (Section 4.1.2 of the paper: the engine is
+ * chosen per layer shape).  The operand format is the caller's choice; on this GPU 8-bit
+ * containers on the tensor cores are faster than bit planes for every size from 64 to 4096 per
+ * dimension and every (w, a), so AUTO never converts between formats, it picks by shape:
+ *   INT8 operands       N <= 8: byte dot products, one warp per weight row;
+ *                       M >= 256, N >= 2048 and at least a round and a half of 256 x 256 tiles
+ *                       on the SM pairs: the CTA-pair tensor-core kernel; else the one-CTA
+ *                       tensor-core kernel
+ *   BITPLANES operands  N <= 16: one warp per weight row over the planes; else the tiled
+ *                       AND/POPC kernel
+ *   FIELDS weights      N <= 16 only: packed weights expanded inside the tensor-core kernel
+ * Returns a qnn_kernel value, or the (negative) qnn_status qnn_qgemm would return.  Host only. */
+typedef enum {
+    QNN_KERNEL_TENSOR = 1, QNN_KERNEL_TENSOR_CTA_PAIR = 2, QNN_KERNEL_BYTES_FEW_COLUMNS = 3,
+    QNN_KERNEL_PLANES_FEW_COLUMNS = 4, QNN_KERNEL_PLANES_TILED = 5, QNN_KERNEL_FIELDS_FEW_COLUMNS = 6
+} qnn_kernel;
+int qnn_qgemm_kernel(const qnn_gemm_desc *d, int has_thresholds);
+
 /* ---- lowering and convolution (Section 3.2) ------------------------------- */
 
 typedef struct {

@@ -10,6 +10,8 @@ qnn_oracle.c   plain C loops: integer GEMM, thresholding, direct convolution,
 oracle.py      ctypes access to the C functions on numpy arrays.
 bitserial.py   Algorithms 1 and 2 of the paper restated on Python integers
                (tiny sizes only; used to pin the GEMM oracle).
+planeskip.py   bit-plane products without the low-order plane pairs (the paper's
+               conclusion: approximate computing from the higher-order bits), numpy int64.
 streamline.py  float batch-norm + quantizer reference and the threshold
                absorption of Section 2.1 (fp64).
 alexnet.py     the AlexNet-shaped layer chain of Section 4.2 built from the above.

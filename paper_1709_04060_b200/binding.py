@@ -33,7 +33,7 @@ QNN_PATH_AUTO, QNN_PATH_BITSERIAL, QNN_PATH_TCGEN05_I8 = 0, 1, 2
 
 EXPORTS = (
     "qnn_packed_ld", "qnn_packed_bytes", "qnn_pack", "qnn_gemm_workspace_bytes",
-    "qnn_gemm_out_bytes", "qnn_qgemm", "qnn_conv_out_h", "qnn_conv_out_w",
+    "qnn_gemm_out_bytes", "qnn_qgemm", "qnn_qgemm_kernel", "qnn_conv_out_h", "qnn_conv_out_w",
     "qnn_conv_lowered_k", "qnn_conv_lowered_bytes", "qnn_conv_workspace_bytes",
     "qnn_conv_out_bytes", "qnn_im2col", "qnn_qconv", "qnn_qconv_static", "qnn_maxpool",
     "qnn_streamline", "qnn_peak_mma_i8", "qnn_peak_popc", "qnn_peak_popc_sink_bytes", "qnn_validate_thresholds", "qnn_device_status", "qnn_launch_count",
@@ -78,6 +78,8 @@ _lib.qnn_gemm_workspace_bytes.restype = _sz
 _lib.qnn_gemm_workspace_bytes.argtypes = [_P(qnn_gemm_desc)]
 _lib.qnn_gemm_out_bytes.restype = _sz
 _lib.qnn_gemm_out_bytes.argtypes = [_P(qnn_gemm_desc), _ci]
+_lib.qnn_qgemm_kernel.restype = _ci
+_lib.qnn_qgemm_kernel.argtypes = [_P(qnn_gemm_desc), _ci]
 _lib.qnn_qgemm.restype = _ci
 _lib.qnn_qgemm.argtypes = [_P(qnn_gemm_desc), _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 for _n in ("qnn_conv_out_h", "qnn_conv_out_w", "qnn_conv_lowered_k"):
@@ -176,6 +178,15 @@ def qnn_gemm_workspace_bytes(d) -> int:
 
 def qnn_gemm_out_bytes(d, has_thresholds: bool) -> int:
     return int(_lib.qnn_gemm_out_bytes(ctypes.byref(d), int(has_thresholds)))
+
+
+QNN_KERNEL_TENSOR, QNN_KERNEL_TENSOR_CTA_PAIR, QNN_KERNEL_BYTES_FEW_COLUMNS = 1, 2, 3
+QNN_KERNEL_PLANES_FEW_COLUMNS, QNN_KERNEL_PLANES_TILED, QNN_KERNEL_FIELDS_FEW_COLUMNS = 4, 5, 6
+
+
+def qnn_qgemm_kernel(d, has_thresholds: bool = True) -> int:
+    """The kernel qnn_qgemm would run for this problem (a QNN_KERNEL_* value, or a negative status)."""
+    return _lib.qnn_qgemm_kernel(ctypes.byref(d), int(has_thresholds))
 
 
 def qnn_qgemm(d, W, A, thr, out, workspace=None, workspace_bytes=0, stream=None) -> int:

@@ -156,6 +156,17 @@ size_t qnn_gemm_out_bytes(const qnn_gemm_desc *d, int has_thresholds) {
     return 0;
 }
 
+int qnn_qgemm_kernel(const qnn_gemm_desc *d, int has_thresholds) {
+    int path = 0;
+    const qnn_status st = check_gemm_desc(d, has_thresholds != 0, &path);
+    if (st != QNN_OK) return (int)st;
+    if (d->w_fmt == QNN_FMT_FIELDS) return QNN_KERNEL_FIELDS_FEW_COLUMNS;
+    if (d->path == QNN_PATH_AUTO && d->w_fmt == QNN_FMT_INT8 && gemv_i8_fits(d)) return QNN_KERNEL_BYTES_FEW_COLUMNS;
+    if (path == QNN_PATH_TCGEN05_I8) return gemm_tc_uses_pair_kernel(d) ? QNN_KERNEL_TENSOR_CTA_PAIR : QNN_KERNEL_TENSOR;
+    if (gemv_planes_fits(d)) return QNN_KERNEL_PLANES_FEW_COLUMNS;
+    return QNN_KERNEL_PLANES_TILED;
+}
+
 qnn_status qnn_qgemm(const qnn_gemm_desc *d, const void *W, const void *A, const int32_t *thr,
                      void *out, void *workspace, size_t workspace_bytes, void *stream) {
     (void)workspace; (void)workspace_bytes;

@@ -74,6 +74,7 @@ qnn_status gemv_fields_launch(const qnn_gemm_desc *d, const void *W, const void 
                               const int32_t *thr, void *out, cudaStream_t s);
 qnn_status gemm_tc_launch(const qnn_gemm_desc *d, const void *W, const void *A,
                           const int32_t *thr, void *out, cudaStream_t s);
+bool gemm_tc_uses_pair_kernel(const qnn_gemm_desc *d);
 qnn_status gemm_tc_conv_launch(const qnn_conv_desc *cv, const qnn_gemm_desc *g, const void *W, const void *in,
                                const int32_t *thr, void *out, cudaStream_t s);
 qnn_status gemm_tc_lower_launch(const qnn_conv_desc *cv, const qnn_gemm_desc *g, const void *W, const void *in,

@@ -269,25 +269,29 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams &p, const int *thr
     if (OUT_BITS >= 3) {
         // bisection over the channel's sorted thresholds: the row of NT words sits in NT
         // distinct banks, so lanes that look at different slots do not conflict
+        // Sixteen channels' searches advance together: a probe's load takes 100+ cycles while the
+        // tensor pipe reads shared memory, and only independent chains hide that.
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
+        for (int g = 0; g < 2; ++g) {
             // the search position is carried as a pointer (row + count): every probe is a load at a
             // constant offset from it, and a step is load, compare, conditional add
-            const int *pos[8];
-            int c[8], t[8];
+            const int *pos[16];
+            int c[16], t[16];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) pos[e] = thr_c + (8 * g + e) * NT;
+            for (int e = 0; e < 16; ++e) pos[e] = thr_c + (16 * g + e) * NT;
 #pragma unroll
             for (int step = NT / 2; step >= 1; step >>= 1) {
 #pragma unroll
-                for (int e = 0; e < 8; ++e) t[e] = pos[e][step - 1];
+                for (int e = 0; e < 16; ++e) t[e] = pos[e][step - 1];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) pos[e] += (acc[8 * g + e] >= t[e]) ? step : 0;
+                for (int e = 0; e < 16; ++e) pos[e] += (acc[16 * g + e] >= t[e]) ? step : 0;
             }
 #pragma unroll
-            for (int e = 0; e < 8; ++e) c[e] = (int)(pos[e] - (thr_c + (8 * g + e) * NT));
-            packed[2 * g] = (uint32_t)c[0] | ((uint32_t)c[1] << 8) | ((uint32_t)c[2] << 16) | ((uint32_t)c[3] << 24);
-            packed[2 * g + 1] = (uint32_t)c[4] | ((uint32_t)c[5] << 8) | ((uint32_t)c[6] << 16) | ((uint32_t)c[7] << 24);
+            for (int e = 0; e < 16; ++e) c[e] = (int)(pos[e] - (thr_c + (16 * g + e) * NT));
+#pragma unroll
+            for (int v = 0; v < 4; ++v)
+                packed[4 * g + v] = (uint32_t)c[4 * v] | ((uint32_t)c[4 * v + 1] << 8) | ((uint32_t)c[4 * v + 2] << 16) |
+                                    ((uint32_t)c[4 * v + 3] << 24);
         }
     } else if (p.fp_count) {
         // NT == 4: one float4 of thresholds per channel
@@ -871,40 +875,6 @@ struct Tc2Smem {
     int abort_flag;
 };
 
-// Work distribution of the CTA-pair kernel.  The output is cut into stripes of 256 pixels, a
-// stripe into units of 64 channels; the units of all stripes, in order, are dealt to the SM
-// pairs as contiguous ranges of (almost) equal length, and a pair cuts its range into tiles of
-// up to four units (256 channels) of about equal width that do not cross a stripe.  An MMA's
-// time is proportional to the tile width from 128 channels up, so every pair gets the same
-// amount of work whatever the ratio of tiles to pairs (256 x 256 tiles dealt round robin left
-// 3.46 rounds of work taking 4 rounds of time at 4096^3).  Every role of the kernel walks the
-// same sequence.
-constexpr int T2_UNIT = 64;
-struct PairSched {
-    long long u, u_end;
-    int U;                      // units per stripe
-    __device__ PairSched(const TcParams &p, int pair, int num_pairs) {
-        U = (p.M + T2_UNIT - 1) / T2_UNIT;
-        const long long total = (long long)p.tiles_p * U;
-        u = total * pair / num_pairs;
-        u_end = total * (pair + 1) / num_pairs;
-    }
-    // next tile: first pixel, first channel, width in channels; false when the range is used up
-    __device__ bool next(int &p0, int &c0, int &bn) {
-        if (u >= u_end) return false;
-        const long long stripe = u / U;
-        const int cu = (int)(u - stripe * U);
-        long long seg_end = (stripe + 1) * U;
-        if (seg_end > u_end) seg_end = u_end;
-        const int rem = (int)(seg_end - u);
-        const int k = (rem + 3) >> 2;                    // tiles left in this stripe segment
-        const int w = (rem + k - 1) / k;                 // widths differ by at most one unit
-        p0 = (int)stripe * 256; c0 = cu * T2_UNIT; bn = w * T2_UNIT;
-        u += w;
-        return true;
-    }
-};
-
 template <int OUT_MODE, int OUT_BITS>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_constant__ CUtensorMap map_wgt,
@@ -940,19 +910,16 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_const
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint32_t tmem_base = sm.tmem_base;
-    PairSched sched(p, pair, num_pairs);
-    int t_p0, t_c0, t_bn;                              // the current tile of this role
+    const int num_tiles = p.tiles_p * p.tiles_c;       // tiles of 256 pixels x 256 channels
 
     if (warp == 0) {
         // ---------------------------------------- producer (one per CTA, own halves)
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            while (ok && sched.next(t_p0, t_c0, t_bn)) {
-                // this CTA's 128 pixels and its half of the tile's channels (the copy always brings
-                // 128 weight rows; a narrower tile uses the first bn / 2 of them)
-                const int p0 = t_p0 + (int)rank * 128;
-                const int c0 = t_c0 + (int)rank * (t_bn >> 1);
+            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+                const int p0 = (tile % p.tiles_p) * 256 + (int)rank * 128;
+                const int c0 = (tile / p.tiles_p) * T2_BN + (int)rank * 128;
                 for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
                     const int s = it % T2_STAGES;
                     const uint32_t ph = (it / T2_STAGES) & 1;
@@ -970,12 +937,11 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_const
         if (lane == 0 && rank == 0) {
             uint32_t it = 0, tcount = 0;
             bool ok = true;
-            for (; ok && sched.next(t_p0, t_c0, t_bn); ++tcount) {
+            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs, ++tcount) {
                 const uint32_t buf = tcount & 1, acc_ph = (tcount >> 1) & 1;
                 if (!(ok = mbar_wait(&sm.tmem_empty[buf], acc_ph ^ 1, abort_flag))) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * T2_BN;
-                const uint32_t idesc = p.idesc | ((uint32_t)(t_bn >> 3) << 17);      // MMA N = the tile's width
                 for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
                     const int s = it % T2_STAGES;
                     const uint32_t ph = (it / T2_STAGES) & 1;
@@ -985,7 +951,7 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_const
                     const uint64_t db = umma_smem_desc(smem_u32(sm.wgt[s]));
 #pragma unroll
                     for (int kk = 0; kk < TC_BK / 32; ++kk)
-                        umma_i8_pair(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (kb | kk) != 0);
+                        umma_i8_pair(d_tmem, da + 2 * kk, db + 2 * kk, p.idesc, (kb | kk) != 0);
                     // free the stage in both CTAs
                     umma_commit_pair(map_to_cta(smem_u32(&sm.empty[s]), 0));
                     umma_commit_pair(map_to_cta(smem_u32(&sm.empty[s]), 1));
@@ -1001,18 +967,21 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_const
         // ------------------------------------ threshold stager (all 256 channels of the tile)
         if (OUT_MODE != OUT_RAW)
             stager_loop<OUT_BITS, T2_BN>(p, &sm.thr[0][0], sm.thr_full, sm.thr_empty, lane, abort_flag,
-                                         [&](uint32_t, int &c0, int &bn) {           // called once per tile, in order
-                                             int p0;
-                                             return sched.next(p0, c0, bn);
+                                         [&](uint32_t i, int &c0, int &bn) {
+                                             const long long tile = pair + (long long)i * num_pairs;
+                                             if (tile >= num_tiles) return false;
+                                             c0 = (int)(tile / p.tiles_p) * T2_BN; bn = T2_BN;
+                                             return true;
                                          });
     } else {
         // ----------------------------- epilogue (each CTA: its 128 pixels, all 256 channels)
         uint32_t tcount = 0;
-        for (; sched.next(t_p0, t_c0, t_bn); ++tcount) {
+        for (int tile = pair; tile < num_tiles; tile += num_pairs, ++tcount) {
+            const int p0 = (tile % p.tiles_p) * 256 + (int)rank * 128, c0 = (tile / p.tiles_p) * T2_BN;
             const uint32_t buf = tcount & 1, acc_ph = (tcount >> 1) & 1;
             if (!epilogue_tile<OUT_MODE, OUT_BITS>(p, sm.thr[buf], &sm.thr_full[buf], &sm.thr_empty[buf], acc_ph,
-                                                   &sm.tmem_full[buf], acc_ph, tmem_base + buf * T2_BN, t_bn,
-                                                   t_p0 + (int)rank * 128, t_c0, -1, TcExchange{}, warp, lane, abort_flag))
+                                                   &sm.tmem_full[buf], acc_ph, tmem_base + buf * T2_BN, T2_BN,
+                                                   p0, c0, -1, TcExchange{}, warp, lane, abort_flag))
                 break;
             if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&sm.tmem_empty[buf]), 0));
         }
@@ -1157,10 +1126,9 @@ static qnn_status launch_pair_cfg(const CUtensorMap &ma, const CUtensorMap &mw, 
             return QNN_ERR_CUDA;
         attr_done[dev] = true;
     }
-    // one SM pair per 64-channel unit of work at most (see PairSched)
-    const long long units = (long long)p.tiles_p * ceil_div(p.M, T2_UNIT);
+    const int tiles = p.tiles_p * p.tiles_c;
     const int max_pairs = sm_count() / 2;
-    const int pairs = units < max_pairs ? (int)units : max_pairs;
+    const int pairs = tiles < max_pairs ? tiles : max_pairs;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(TC_THREADS);
     cfg.dynamicSmemBytes = smem; cfg.stream = s;
@@ -1270,6 +1238,8 @@ static bool tc_plan(const qnn_gemm_desc *d, int sms, int num_kb, TcPlan *pl) {
     return true;
 }
 
+bool gemm_tc_uses_pair_kernel(const qnn_gemm_desc *d) { return choose_pair_kernel(d, sm_count()); }
+
 // cv != nullptr: implicit convolution, A is the feature map (see TcParams); d is the lowered GEMM.
 static qnn_status tc_launch(const qnn_gemm_desc *d, const qnn_conv_desc *cv, const void *W, const void *A,
                             const int32_t *thr, void *out, cudaStream_t s) {
@@ -1306,7 +1276,7 @@ static qnn_status tc_launch(const qnn_gemm_desc *d, const qnn_conv_desc *cv, con
         if (!make_map(&ma, A, d->N, d->K, ld, TC_BP) || !make_map(&mw, W, d->M, d->K, ld, 128)) return QNN_ERR_CUDA;
         p.tiles_p = ceil_div(d->N, 256); p.tiles_c = ceil_div(d->M, T2_BN);
         p.units = p.full_units = p.tiles_p * p.tiles_c;
-        p.idesc = idesc_base | ((uint32_t)(256 >> 4) << 24);          // the kernel adds each tile's N
+        p.idesc = idesc_base | ((uint32_t)(T2_BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
         return launch_pair_out(mode, d->out_bits, ma, mw, p, s);
     }
     TcPlan pl;
