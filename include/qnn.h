@@ -123,6 +123,14 @@ typedef struct {
     int path;             /* qnn_path; AUTO selects by operand format, and for a
                              handful of columns (N <= 16 bit planes, N <= 8
                              bytes) the one-warp-per-weight-row kernels       */
+    int skip_planes;      /* 0: the exact product.  s > 0 (BITPLANES operands only):
+                             the bit-plane pairs (i, j) with i + j < s are left out
+                             of sum_i sum_j +-2^(i+j) W[i].A[j] -- the approximate
+                             product from the higher-order bits that the paper's
+                             conclusion names; it differs from the exact one by at
+                             most K * sum_{i+j<s} 2^(i+j), and the bit-serial kernels
+                             skip the AND/POPC work of those pairs.  A BIPOLAR
+                             operand counts as one plane (index 0).               */
 } qnn_gemm_desc;
 
 /* Scratch bytes qnn_qgemm needs for this problem (may be 0).  Host only. */

@@ -48,7 +48,7 @@ class qnn_pack_desc(ctypes.Structure):
 class qnn_gemm_desc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in (
         "M", "N", "K", "w_bits", "a_bits", "out_bits", "w_enc", "a_enc",
-        "w_fmt", "a_fmt", "out_fmt", "path")]
+        "w_fmt", "a_fmt", "out_fmt", "path", "skip_planes")]
 
 
 class qnn_conv_desc(ctypes.Structure):
@@ -312,8 +312,8 @@ def pack(logical: torch.Tensor, bits: int, enc: int, fmt: int, stream=None) -> t
 
 
 def gemm_desc(M, N, K, w_bits, a_bits, out_bits, w_enc, a_enc, fmt, out_fmt,
-              path=QNN_PATH_AUTO) -> qnn_gemm_desc:
-    return qnn_gemm_desc(M, N, K, w_bits, a_bits, out_bits, w_enc, a_enc, fmt, fmt, out_fmt, path)
+              path=QNN_PATH_AUTO, skip_planes=0) -> qnn_gemm_desc:
+    return qnn_gemm_desc(M, N, K, w_bits, a_bits, out_bits, w_enc, a_enc, fmt, fmt, out_fmt, path, skip_planes)
 
 
 def qgemm(d: qnn_gemm_desc, W, A, thr, out=None, stream=None) -> torch.Tensor:

@@ -31,6 +31,9 @@ static qnn_status check_gemm_desc(const qnn_gemm_desc *d, bool has_thr, int *pat
     if (!(valid_fmt(d->w_fmt) || d->w_fmt == QNN_FMT_FIELDS) || !valid_fmt(d->a_fmt)) return QNN_ERR_INVALID_ARG;
     if (d->w_enc < 0 || d->w_enc > 2 || d->a_enc < 0 || d->a_enc > 2) return QNN_ERR_INVALID_ARG;
     if (d->path < QNN_PATH_AUTO || d->path > QNN_PATH_TCGEN05_I8) return QNN_ERR_INVALID_ARG;
+    if (d->skip_planes < 0) return QNN_ERR_INVALID_ARG;
+    // leaving plane pairs out is a notion of the bit-plane formulation only
+    if (d->skip_planes > 0 && (d->w_fmt != QNN_FMT_BITPLANES || d->a_fmt != QNN_FMT_BITPLANES)) return QNN_ERR_UNSUPPORTED;
     if (has_thr) {
         if (d->out_bits < 1 || d->out_bits > 4) return QNN_ERR_INVALID_ARG;
         if (!valid_fmt(d->out_fmt)) return QNN_ERR_INVALID_ARG;
@@ -92,6 +95,7 @@ static void conv_to_gemm(const qnn_conv_desc *d, qnn_gemm_desc *g) {
     g->w_enc = d->w_enc; g->a_enc = d->a_enc;
     g->w_fmt = d->fmt; g->a_fmt = d->fmt; g->out_fmt = d->out_fmt;
     g->path = d->path;
+    g->skip_planes = 0;
 }
 
 }  // namespace qnn

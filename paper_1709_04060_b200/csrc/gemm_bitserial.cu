@@ -82,27 +82,31 @@ qgemm_bitserial_kernel(const BsParams p) {
 
 #pragma unroll 2
         for (int cc = 0; cc < BS_KT; ++cc) {
-            uint32_t wv[2][WB];
+            uint32_t wv[2][WB], av[BS_TN][AB];
 #pragma unroll
             for (int t = 0; t < 2; ++t)
 #pragma unroll
                 for (int i = 0; i < WB; ++i) wv[t][i] = Ws[i][lane + 32 * t][cc];
 #pragma unroll
-            for (int nn = 0; nn < BS_TN; ++nn) {
-                uint32_t av[AB];
+            for (int nn = 0; nn < BS_TN; ++nn)
 #pragma unroll
-                for (int j = 0; j < AB; ++j) av[j] = As[j][warp * BS_TN + nn][cc];
+                for (int j = 0; j < AB; ++j) av[nn][j] = As[j][warp * BS_TN + nn][cc];
+            // plane pair outermost: a pair that is left out (coefficient 0, uniform) costs one branch
 #pragma unroll
-                for (int t = 0; t < 2; ++t)
+            for (int i = 0; i < WB; ++i)
 #pragma unroll
-                    for (int i = 0; i < WB; ++i)
+                for (int j = 0; j < AB; ++j) {
+                    const int cf = p.coef[i][j];
+                    if (cf == 0) continue;
 #pragma unroll
-                        for (int j = 0; j < AB; ++j) {
-                            const uint32_t x = (MODE == BS_BOTH_BIPOLAR) ? (wv[t][i] ^ av[j])
-                                                                          : (wv[t][i] & av[j]);
-                            acc[t][nn] += p.coef[i][j] * __popc(x);
+                    for (int nn = 0; nn < BS_TN; ++nn)
+#pragma unroll
+                        for (int t = 0; t < 2; ++t) {
+                            const uint32_t x = (MODE == BS_BOTH_BIPOLAR) ? (wv[t][i] ^ av[nn][j])
+                                                                          : (wv[t][i] & av[nn][j]);
+                            acc[t][nn] += cf * __popc(x);
                         }
-            }
+                }
         }
         __syncthreads();
     }
@@ -207,15 +211,21 @@ qnn_status gemm_bitserial_launch(const qnn_gemm_desc *d, const void *W, const vo
     for (int i = 0; i < 4; ++i) p.corr[i] = 0;
     for (int i = 0; i < 4; ++i)
         for (int j = 0; j < 4; ++j) p.coef[i][j] = cw[i] * ca[j];
+    // plane pairs (i, j) with i + j < skip_planes are left out (a bipolar operand is plane 0)
+    const int skip = d->skip_planes;
+    for (int i = 0; i < 4; ++i)
+        for (int j = 0; j < 4; ++j)
+            if (i + j < skip) p.coef[i][j] = 0;
     bool ok;
     if (wb && ab) {
-        p.coef[0][0] = -2;
+        p.coef[0][0] = skip > 0 ? 0 : -2;
+        if (skip > 0) p.K = 0;                       // the pair's K - 2 popc(xor) goes as a whole
         ok = dispatch_bits<BS_BOTH_BIPOLAR>(1, 1, p, s);
     } else if (wb) {
-        for (int j = 0; j < 4; ++j) { p.coef[0][j] = 2 * ca[j]; p.corr[j] = ca[j]; }
+        for (int j = 0; j < 4; ++j) { p.coef[0][j] = j < skip ? 0 : 2 * ca[j]; p.corr[j] = j < skip ? 0 : ca[j]; }
         ok = dispatch_bits<BS_W_BIPOLAR>(1, d->a_bits, p, s);
     } else if (ab) {
-        for (int i = 0; i < 4; ++i) { p.coef[i][0] = 2 * cw[i]; p.corr[i] = cw[i]; }
+        for (int i = 0; i < 4; ++i) { p.coef[i][0] = i < skip ? 0 : 2 * cw[i]; p.corr[i] = i < skip ? 0 : cw[i]; }
         ok = dispatch_bits<BS_A_BIPOLAR>(d->w_bits, 1, p, s);
     } else {
         ok = dispatch_bits<BS_REGULAR>(d->w_bits, d->a_bits, p, s);

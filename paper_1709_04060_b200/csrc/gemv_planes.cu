@@ -93,6 +93,7 @@ gemv_planes_kernel(const GvParams p) {
                                 gv_smem + (j * GV_COLS + c) * p.kw_pad + 4 * q);
 #pragma unroll
                             for (int i = 0; i < WB; ++i) {
+                                if (p.coef[i][j] == 0) continue;   // a plane pair that is left out (uniform)
                                 int cnt;
                                 if (MODE == GV_BOTH_BIPOLAR)
                                     cnt = __popc(wv[i].x ^ av.x) + __popc(wv[i].y ^ av.y) +
@@ -123,6 +124,7 @@ gemv_planes_kernel(const GvParams p) {
                             const uint32_t av = gv_smem[(j * GV_COLS + c) * p.kw_pad + d];
 #pragma unroll
                             for (int i = 0; i < WB; ++i) {
+                                if (p.coef[i][j] == 0) continue;
                                 const uint32_t x = (MODE == GV_BOTH_BIPOLAR) ? (wv[i] ^ av) : (wv[i] & av);
                                 acc[c] += p.coef[i][j] * __popc(x);
                             }
@@ -246,15 +248,21 @@ qnn_status gemv_planes_launch(const qnn_gemm_desc *d, const void *W, const void 
     const int row_blocks = ceil_div(d->M, GV_THREADS / 32);
     const int max_blocks = sm_count() * 8;
     dim3 grid(row_blocks < max_blocks ? row_blocks : max_blocks, ceil_div(d->N, GV_COLS));
+    // plane pairs (i, j) with i + j < skip_planes are left out (a bipolar operand is plane 0)
+    const int skip = d->skip_planes;
+    for (int i = 0; i < 4; ++i)
+        for (int j = 0; j < 4; ++j)
+            if (i + j < skip) p.coef[i][j] = 0;
     bool ok;
     if (wb && ab) {
-        p.coef[0][0] = -2;
+        p.coef[0][0] = skip > 0 ? 0 : -2;
+        if (skip > 0) p.K = 0;                       // the pair's K - 2 popc(xor) goes as a whole
         ok = gv_dispatch<GV_BOTH_BIPOLAR>(1, 1, p, grid, smem, s);
     } else if (wb) {
-        for (int j = 0; j < 4; ++j) { p.coef[0][j] = 2 * ca[j]; p.corr[j] = ca[j]; }
+        for (int j = 0; j < 4; ++j) { p.coef[0][j] = j < skip ? 0 : 2 * ca[j]; p.corr[j] = j < skip ? 0 : ca[j]; }
         ok = gv_dispatch<GV_W_BIPOLAR>(1, d->a_bits, p, grid, smem, s);
     } else if (ab) {
-        for (int i = 0; i < 4; ++i) { p.coef[i][0] = 2 * cw[i]; p.corr[i] = cw[i]; }
+        for (int i = 0; i < 4; ++i) { p.coef[i][0] = i < skip ? 0 : 2 * cw[i]; p.corr[i] = i < skip ? 0 : cw[i]; }
         ok = gv_dispatch<GV_A_BIPOLAR>(d->w_bits, 1, p, grid, smem, s);
     } else {
         ok = gv_dispatch<GV_REGULAR>(d->w_bits, d->a_bits, p, grid, smem, s);

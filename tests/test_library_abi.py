@@ -145,3 +145,29 @@ def test_argument_validation_without_launch(qb):
 
     pl = qb.qnn_pool_desc(1, 2, 2, 16, 3, 2, 2, 1)
     assert qb.qnn_maxpool(pl, P, P, stream=0) == qb.QNN_ERR_INVALID_ARG
+
+
+def test_kernel_choice_follows_the_documented_rule(qb):
+    """qnn_qgemm_kernel (host only): the shape-driven choice documented in qnn.h -- the operand
+    format is the caller's, the kernel follows from the shape (size sweep of Section 4.1.2)."""
+    I8, PL, FL = qb.QNN_FMT_INT8, qb.QNN_FMT_BITPLANES, qb.QNN_FMT_FIELDS
+
+    def k(M, N, K, w_fmt, a_fmt, path=0, w=2, a=2):
+        d = qb.qnn_gemm_desc(M, N, K, w, a, 2, 1, 0, w_fmt, a_fmt, I8, path, 0)
+        return qb.qnn_qgemm_kernel(d, True)
+
+    assert k(4096, 4096, 4096, I8, I8) == qb.QNN_KERNEL_TENSOR_CTA_PAIR
+    assert k(8192, 8192, 8192, I8, I8) == qb.QNN_KERNEL_TENSOR_CTA_PAIR
+    assert k(4096, 1024, 4096, I8, I8) == qb.QNN_KERNEL_TENSOR            # fewer than 2048 columns
+    assert k(128, 4096, 4096, I8, I8) == qb.QNN_KERNEL_TENSOR             # fewer than 256 channels
+    assert k(64, 256, 576, I8, I8) == qb.QNN_KERNEL_TENSOR                # config 1
+    assert k(8192, 1, 8192, I8, I8) == qb.QNN_KERNEL_BYTES_FEW_COLUMNS
+    assert k(8192, 8, 8192, I8, I8) == qb.QNN_KERNEL_BYTES_FEW_COLUMNS
+    assert k(8192, 16, 8192, I8, I8) == qb.QNN_KERNEL_TENSOR
+    assert k(8192, 8, 8192, I8, I8, path=2) == qb.QNN_KERNEL_TENSOR       # path forced
+    assert k(8192, 16, 8192, PL, PL) == qb.QNN_KERNEL_PLANES_FEW_COLUMNS
+    assert k(8192, 17, 8192, PL, PL) == qb.QNN_KERNEL_PLANES_TILED
+    assert k(64, 256, 576, PL, PL) == qb.QNN_KERNEL_PLANES_TILED
+    assert k(8192, 16, 8192, FL, I8) == qb.QNN_KERNEL_FIELDS_FEW_COLUMNS
+    assert k(8192, 17, 8192, FL, I8) == qb.QNN_ERR_UNSUPPORTED
+    assert k(64, 64, 64, I8, PL) == qb.QNN_ERR_UNSUPPORTED                # mixed formats
