@@ -699,14 +699,14 @@ def run_extras(args):
         c = synth.gemm_case(5000 + bits, M, 16, K, bits, bits)
         Wd = qb.to_device_logical(c.W, c.w_enc)
         thr = torch.from_numpy(c.thr).cuda()
-        for fmt, name in ((PL, "bitplanes"), (I8, "int8")):
+        for fmt, afmt, name in SKINNY_FORMATS(qb):
             Wp = qb.pack(Wd, bits, c.w_enc, fmt)
             copies = max(2, int(300e6 // Wp.numel()) + 1)          # > 2 x L2 in rotation
             Wrot = [Wp] + [Wp.clone() for _ in range(copies - 1)]
             for N in (1, 4, 16):
                 Ad = qb.to_device_logical(c.At[:N], c.a_enc)
-                Ap = qb.pack(Ad, bits, c.a_enc, fmt)
-                d = qb.gemm_desc(M, N, K, bits, bits, bits, c.w_enc, c.a_enc, fmt, I8)
+                Ap = qb.pack(Ad, bits, c.a_enc, afmt)
+                d = qb.qnn_gemm_desc(M, N, K, bits, bits, bits, c.w_enc, c.a_enc, fmt, afmt, I8, 0)
                 out = torch.empty(qb.qnn_gemm_out_bytes(d, True), dtype=torch.uint8, device="cuda")
                 ms = _time_calls(torch, lambda i: qb.check(qb.qnn_qgemm(d, Wrot[i % copies], Ap, thr, out)),
                                  4 * copies, graph=True)
@@ -843,7 +843,7 @@ def run_shapes(args):
 # dram__bytes_read.sum + dram__bytes_write.sum of one 4096^3 W1A2 launch of the (CTA-pair)
 # tensor-core kernel, from an ncu capture of that launch (the output codes were still in L2 when
 # the capture ended, so the write counter is small).
-TRAFFIC_BYTES_PER_LAUNCH = 33648384 + 79360
+TRAFFIC_BYTES_PER_LAUNCH = 33648640 + 94208
 
 
 def main():

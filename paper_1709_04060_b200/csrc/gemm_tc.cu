@@ -1204,8 +1204,11 @@ static bool tc_plan(const qnn_gemm_desc *d, int sms, int num_kb, TcPlan *pl) {
     const int cand[3] = {256, 128, 32};
     double best_cost = 0.0;
     int bn = 0;
+    const char *force_bn = getenv("QNN_TC_BN");               // "256" | "128" | "32": measurements only
+    const int forced = force_bn ? atoi(force_bn) : 0;
     for (int ci = 0; ci < 3; ++ci) {
         const int b = cand[ci];
+        if (forced && b != forced) continue;
         if (b > 32 && b / 2 >= round_up(d->M, 32)) continue;        // wider than the channels need
         const long long t = (long long)tiles_p * ceil_div(d->M, b);
         const double main_loop = 640.0 * num_kb, epi = 2000.0 * (b >= 64 ? b / 64 : 1);
