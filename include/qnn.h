@@ -224,7 +224,8 @@ qnn_status qnn_im2col(const qnn_conv_desc *d, const void *in, void *lowered, voi
  * M = OC, i.e. a channels-last feature map [B][OH][OW][...].  BIPOLAR
  * activations with pad > 0 are UNSUPPORTED (zero is not representable).
  * The lowered matrix of Section 3.2 is written to `workspace` only where the
- * GEMM kernel cannot form its tiles itself: 8-bit maps are lowered inside the
+ * GEMM kernel cannot form its tiles itself: bit-plane maps are lowered on the fly by the
+ * staging code of the tiled AND/POPC kernel (word-granular, as in Section 3.2); 8-bit maps are lowered inside the
  * kernel (by its tensor-map loader when C and in_pitch are multiples of 16; by
  * lowering warps when pixels are contiguous and either C is not a multiple of
  * 16, pad == 0 and OC <= 128, or C is a multiple of 16 but not of 128 and the

@@ -259,6 +259,12 @@ qnn_status qnn_qconv(const qnn_conv_desc *d, const void *Wpacked, const void *in
         st = gemm_tc_conv_launch(d, &g, Wpacked, in, thr, out, (cudaStream_t)stream);
         if (st != QNN_ERR_UNSUPPORTED) return st;
     }
+    // bit-plane maps on the tiled bit-serial kernel: its staging code lowers on the fly (a handful
+    // of output pixels goes through the lowered matrix and the few-column kernel instead)
+    if (path == QNN_PATH_BITSERIAL && !(explicit_env && explicit_env[0] == '1') && !gemv_planes_fits(&g)) {
+        st = gemm_bitserial_conv_launch(d, &g, Wpacked, in, thr, out, (cudaStream_t)stream);
+        if (st != QNN_ERR_UNSUPPORTED) return st;
+    }
     st = im2col_launch(d, in, workspace, (cudaStream_t)stream);
     if (st != QNN_OK) return st;
     return qnn_qgemm(&g, Wpacked, workspace, thr, out, nullptr, 0, stream);

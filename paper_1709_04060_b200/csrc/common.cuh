@@ -63,6 +63,8 @@ int sm_count();
 qnn_status pack_launch(const qnn_pack_desc *d, const void *logical, void *packed, cudaStream_t s);
 qnn_status gemm_bitserial_launch(const qnn_gemm_desc *d, const void *W, const void *A,
                                  const int32_t *thr, void *out, cudaStream_t s);
+qnn_status gemm_bitserial_conv_launch(const qnn_conv_desc *cv, const qnn_gemm_desc *g, const void *W,
+                                      const void *in, const int32_t *thr, void *out, cudaStream_t s);
 bool gemv_i8_fits(const qnn_gemm_desc *d);
 qnn_status gemv_i8_launch(const qnn_gemm_desc *d, const void *W, const void *A,
                           const int32_t *thr, void *out, cudaStream_t s);

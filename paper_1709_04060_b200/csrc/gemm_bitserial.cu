@@ -32,6 +32,12 @@ struct BsParams {
     int out_bits, out_fmt, ld_out;
     int coef[4][4];        // multiplier of popc(W[i] op A[j])
     int corr[4];           // multiplier of the correction popcounts (modes 1, 2)
+    // Implicit convolution (conv != 0): A is the channel-interleaved bit-plane map
+    // [AB][B][H][W][cw] itself, and the staging code does the lowering of Section 3.2 on the fly:
+    // depth word c of output pixel n is word c % cw of input pixel (oh*stride - pad + kh,
+    // ow*stride - pad + kw), (kh, kw) = tap c / cw in raster order; zero outside the image.
+    int conv, cv_H, cv_W, cv_cw, cv_KW, cv_stride, cv_pad, cv_OW, cv_OHW;
+    long long cv_plane;    // words per plane of the map: B*H*W*cw
 };
 
 enum { BS_REGULAR = 0, BS_W_BIPOLAR = 1, BS_A_BIPOLAR = 2, BS_BOTH_BIPOLAR = 3 };
@@ -55,9 +61,30 @@ qgemm_bitserial_kernel(const BsParams p) {
         for (int nn = 0; nn < BS_TN; ++nn) acc[t][nn] = 0;
     int corr_part[4] = {0, 0, 0, 0};             // rows lr, lr+16, lr+32, lr+48
 
+    // implicit convolution: first tap of the four output pixels this thread stages
+    int cv_ih0[4], cv_iw0[4];
+    long long cv_img[4];
+    if (p.conv) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int n = min(n0 + lr + 16 * q, p.N - 1);
+            const int b = n / p.cv_OHW, rem = n - b * p.cv_OHW, oh = rem / p.cv_OW, ow = rem - oh * p.cv_OW;
+            cv_ih0[q] = oh * p.cv_stride - p.cv_pad;
+            cv_iw0[q] = ow * p.cv_stride - p.cv_pad;
+            cv_img[q] = (long long)b * p.cv_H * p.cv_W * p.cv_cw;
+        }
+    }
+
     for (int kw0 = 0; kw0 < p.kw; kw0 += BS_KT) {
         const int c = kw0 + lc;
         const bool c_ok = c < p.kw;
+        int cv_kh = 0, cv_kw = 0, cv_word = 0;
+        if (p.conv) {
+            const int tap = c / p.cv_cw;
+            cv_word = c - tap * p.cv_cw;
+            cv_kh = tap / p.cv_KW;
+            cv_kw = tap - cv_kh * p.cv_KW;
+        }
 #pragma unroll
         for (int i = 0; i < WB; ++i)
 #pragma unroll
@@ -74,7 +101,13 @@ qgemm_bitserial_kernel(const BsParams p) {
             for (int q = 0; q < 4; ++q) {
                 const int r = lr + 16 * q, n = n0 + r;
                 uint32_t v = 0;
-                if (c_ok && n < p.N) v = p.A[((size_t)j * p.N + n) * p.kw + c];
+                if (p.conv) {
+                    const int ih = cv_ih0[q] + cv_kh, iw = cv_iw0[q] + cv_kw;
+                    if (c_ok && n < p.N && (unsigned)ih < (unsigned)p.cv_H && (unsigned)iw < (unsigned)p.cv_W)
+                        v = p.A[(size_t)j * p.cv_plane + cv_img[q] + ((size_t)ih * p.cv_W + iw) * p.cv_cw + cv_word];
+                } else if (c_ok && n < p.N) {
+                    v = p.A[((size_t)j * p.N + n) * p.kw + c];
+                }
                 As[j][r][lc] = v;
                 if (MODE == BS_W_BIPOLAR) corr_part[q] += p.corr[j] * __popc(v);
             }
@@ -196,10 +229,17 @@ static void plane_coef(int bits, int enc, int *c) {
     for (int i = 0; i < bits; ++i) c[i] = (enc == QNN_ENC_SIGNED && i == bits - 1) ? -(1 << i) : (1 << i);
 }
 
-qnn_status gemm_bitserial_launch(const qnn_gemm_desc *d, const void *W, const void *A,
-                                 const int32_t *thr, void *out, cudaStream_t s) {
+static qnn_status bs_launch(const qnn_gemm_desc *d, const qnn_conv_desc *cv, const void *W, const void *A,
+                            const int32_t *thr, void *out, cudaStream_t s) {
     BsParams p;
     p.W = (const uint32_t *)W; p.A = (const uint32_t *)A; p.thr = thr; p.out = out;
+    p.conv = 0; p.cv_H = p.cv_W = p.cv_cw = p.cv_KW = p.cv_stride = p.cv_OW = p.cv_OHW = 1; p.cv_pad = 0; p.cv_plane = 0;
+    if (cv) {
+        p.conv = 1; p.cv_H = cv->H; p.cv_W = cv->W; p.cv_cw = ceil_div(cv->C, 32); p.cv_KW = cv->KW;
+        p.cv_stride = cv->stride; p.cv_pad = cv->pad;
+        p.cv_OW = qnn_conv_out_w(cv); p.cv_OHW = qnn_conv_out_h(cv) * p.cv_OW;
+        p.cv_plane = (long long)cv->B * cv->H * cv->W * p.cv_cw;
+    }
     p.M = d->M; p.N = d->N; p.K = d->K; p.kw = ceil_div(d->K, 32);
     p.out_bits = thr ? d->out_bits : 0;
     p.out_fmt = d->out_fmt;
@@ -233,6 +273,20 @@ qnn_status gemm_bitserial_launch(const qnn_gemm_desc *d, const void *W, const vo
     if (!ok) return QNN_ERR_UNSUPPORTED;
     count_launch();
     return launch_status();
+}
+
+qnn_status gemm_bitserial_launch(const qnn_gemm_desc *d, const void *W, const void *A,
+                                 const int32_t *thr, void *out, cudaStream_t s) {
+    return bs_launch(d, nullptr, W, A, thr, out, s);
+}
+
+// Convolution on bit-plane maps without a lowered matrix: the tiled kernel's staging code reads
+// the map through the lowering's index arithmetic.  g: the lowered GEMM (N = B*OH*OW,
+// K = 32*KH*KW*ceil(C/32)).
+qnn_status gemm_bitserial_conv_launch(const qnn_conv_desc *cv, const qnn_gemm_desc *g, const void *W,
+                                      const void *in, const int32_t *thr, void *out, cudaStream_t s) {
+    if (cv->fmt != QNN_FMT_BITPLANES) return QNN_ERR_UNSUPPORTED;
+    return bs_launch(g, cv, W, in, thr, out, s);
 }
 
 }  // namespace qnn
