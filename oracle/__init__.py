@@ -8,8 +8,8 @@ Contents
 qnn_oracle.c   plain C loops: integer GEMM, thresholding, direct convolution,
                max-pool (compiled by ``oracle.build``).
 oracle.py      ctypes access to the C functions on numpy arrays.
-bitserial.py   Algorithms 1 and 2 of the paper restated on Python integers
-               (tiny sizes only; used to pin the GEMM oracle).
+bitserial.py   the bit-plane identity of Section 3.1 (Algorithms 1-2) on Python integers,
+               one big integer per plane row (tiny sizes only; pins the GEMM oracle).
 planeskip.py   bit-plane products without the low-order plane pairs (the paper's
                conclusion: approximate computing from the higher-order bits), numpy int64.
 streamline.py  float batch-norm + quantizer reference and the threshold

@@ -1,21 +1,23 @@
-"""Algorithms 1 and 2 of the paper on Python integers (TEST INFRASTRUCTURE ONLY).
+"""The bit-plane identity of Section 3.1 on Python integers (TEST INFRASTRUCTURE ONLY).
 
-A slow restatement, for tiny matrices, of the bit-serial formulation of
-Section 3.1: operands are split into bit planes, each plane is packed into
-words along the depth dimension, and every pair of planes contributes
-``+-2^(i+j) * popcount(W(r,d) & A(c,d))``.  It exists to pin the plain integer
-GEMM oracle to the identity the paper states, and to spell out the reading of
-the encodings the paper leaves open:
+Section 3.1 (Algorithms 1-2) states that a few-bit integer product is a weighted sum of binary
+products of bit planes, each binary product being a population count of an AND along the depth:
 
-* UNSIGNED operand: every plane has weight +2^i.
-* SIGNED (two's complement) operand: the most significant plane has weight
-  -2^(bits-1) (Algorithm 2's sgnW / sgnA).
-* BIPOLAR operand (1 bit, bit 1 -> +1, bit 0 -> -1): w = 2b - 1, so
-  ``w.a = 2*(b.a) - sum(a)``; two bipolar operands give the XNOR-popcount form
-  ``K - 2*popcount(a xor b)`` quoted in Section 3.1.
+    W . A = sum_i sum_j c_i^W c_j^A * popcount(W[i] row  AND  A[j] column).
+
+This module restates that identity for tiny matrices so that the plain integer GEMM oracle can be
+pinned to it.  It is organised around the identity, not around a kernel: every row of a plane is
+ONE arbitrary-precision Python integer (bit k = element k), so a binary dot product is a single
+``popcount(x & y)`` with no word loop, and the plane weights come from a small table.  It also
+spells out the reading of the encodings the paper leaves open:
+
+* UNSIGNED operand of b bits: planes 0..b-1, weight +2^i each.
+* SIGNED (two's complement): the same planes, the top one with weight -2^(b-1) (the sign rule of
+  Algorithm 2).
+* BIPOLAR (1 bit, bit 1 -> +1, bit 0 -> -1): x = 2 beta - 1 with beta the bit, so
+  x . y = 2 (beta . y) - sum(y); two bipolar operands give the XNOR-popcount form
+  K - 2 popcount(beta_x xor beta_y) quoted in Section 3.1.
 """
-
-WORDSIZE = 32
 
 UNSIGNED, SIGNED, BIPOLAR = 0, 1, 2
 
@@ -24,80 +26,47 @@ def popcount(x: int) -> int:
     return bin(x).count("1")
 
 
-def pack_planes(X, bits: int, enc: int):
-    """X: list of rows of logical ints -> planes[i][row][d] of WORDSIZE-bit words.
-
-    Element k of a row lands in word k // WORDSIZE at bit k % WORDSIZE; the
-    last word is padded with zero bits."""
-    planes = []
-    for i in range(bits):
-        plane = []
-        for row in X:
-            nwords = (len(row) + WORDSIZE - 1) // WORDSIZE
-            words = [0] * nwords
-            for k, v in enumerate(row):
-                if enc == BIPOLAR:
-                    assert v in (-1, 1)
-                    bit = 1 if v == 1 else 0
-                else:
-                    bit = (int(v) >> i) & 1  # two's complement bit i
-                words[k // WORDSIZE] |= bit << (k % WORDSIZE)
-            plane.append(words)
-        planes.append(plane)
-    return planes
+def plane_weights(bits: int, enc: int):
+    """Weight of each bit plane of an operand (a BIPOLAR operand has its bit as only plane)."""
+    if enc == BIPOLAR:
+        return [1]
+    return [(-(1 << i) if (enc == SIGNED and i == bits - 1) else (1 << i)) for i in range(bits)]
 
 
-def binary_gemm(Wp, Ap, res, alpha: int):
-    """Algorithm 1: res[r][c] += alpha * popcount(W(r,d) & A(c,d)) over depth words."""
-    rows, cols = len(Wp), len(Ap)
-    for r in range(rows):
-        for c in range(cols):
-            for d in range(len(Wp[r])):
-                res[r][c] += alpha * popcount(Wp[r][d] & Ap[c][d])
+def row_planes(row, bits: int, enc: int):
+    """One Python integer per plane: bit k of plane i is bit i of element k (the bit itself for a
+    BIPOLAR element: +1 -> 1, -1 -> 0)."""
+    n_planes = 1 if enc == BIPOLAR else bits
+    out = [0] * n_planes
+    for k, v in enumerate(row):
+        v = int(v)
+        if enc == BIPOLAR:
+            assert v in (-1, 1)
+            out[0] |= (1 if v == 1 else 0) << k
+        else:
+            for i in range(bits):
+                out[i] |= ((v >> i) & 1) << k            # >> on a negative int: two's-complement bits
+    return out
+
+
+def bitserial_dot(w_planes, a_planes, cw, ca, w_enc, a_enc, K: int, a_sum: int, w_sum: int) -> int:
+    """One accumulator from the planes of a weight row and of an activation column."""
+    if w_enc == BIPOLAR and a_enc == BIPOLAR:
+        return K - 2 * popcount(w_planes[0] ^ a_planes[0])
+    if w_enc == BIPOLAR:                                  # (2 beta - 1) . a = 2 (beta . a) - sum(a)
+        return 2 * sum(c * popcount(w_planes[0] & aj) for c, aj in zip(ca, a_planes)) - a_sum
+    if a_enc == BIPOLAR:
+        return 2 * sum(c * popcount(wi & a_planes[0]) for c, wi in zip(cw, w_planes)) - w_sum
+    return sum(ci * cj * popcount(wi & aj) for ci, wi in zip(cw, w_planes) for cj, aj in zip(ca, a_planes))
 
 
 def bitserial_gemm(W, At, w_bits, a_bits, w_enc, a_enc):
-    """Algorithm 2 generalised to per-operand encodings. W[M][K], At[N][K] lists."""
-    M, N = len(W), len(At)
-    K = len(W[0]) if M else 0
-    res = [[0] * N for _ in range(M)]
-
-    if w_enc == BIPOLAR and a_enc == BIPOLAR:
-        wp = pack_planes(W, 1, BIPOLAR)[0]
-        ap = pack_planes(At, 1, BIPOLAR)[0]
-        for r in range(M):
-            for c in range(N):
-                diff = sum(popcount(wp[r][d] ^ ap[c][d]) for d in range(len(wp[r])))
-                res[r][c] = K - 2 * diff
-        return res
-
-    if w_enc == BIPOLAR or a_enc == BIPOLAR:
-        # x = 2b - 1 on the bipolar side: x.y = 2*(b.y) - sum(y)
-        if w_enc == BIPOLAR:
-            Bp = pack_planes(W, 1, BIPOLAR)
-            Op = pack_planes(At, a_bits, a_enc)
-            o_bits, o_enc, other = a_bits, a_enc, At
-        else:
-            Bp = pack_planes(At, 1, BIPOLAR)
-            Op = pack_planes(W, w_bits, w_enc)
-            o_bits, o_enc, other = w_bits, w_enc, W
-        for j in range(o_bits):
-            sgn = -1 if (o_enc == SIGNED and j == o_bits - 1) else 1
-            if w_enc == BIPOLAR:
-                binary_gemm(Bp[0], Op[j], res, 2 * sgn * (1 << j))
-            else:
-                binary_gemm(Op[j], Bp[0], res, 2 * sgn * (1 << j))
-        sums = [sum(int(v) for v in row) for row in other]
-        for r in range(M):
-            for c in range(N):
-                res[r][c] -= sums[c] if w_enc == BIPOLAR else sums[r]
-        return res
-
-    Wp = pack_planes(W, w_bits, w_enc)
-    Ap = pack_planes(At, a_bits, a_enc)
-    for i in range(w_bits):
-        for j in range(a_bits):
-            sgn_w = -1 if (w_enc == SIGNED and i == w_bits - 1) else 1
-            sgn_a = -1 if (a_enc == SIGNED and j == a_bits - 1) else 1
-            binary_gemm(Wp[i], Ap[j], res, sgn_w * sgn_a * (1 << (i + j)))
-    return res
+    """acc[m][n] by the bit-plane identity.  W[M][K], At[N][K]: lists of rows of logical ints."""
+    K = len(W[0]) if W else 0
+    cw, ca = plane_weights(w_bits, w_enc), plane_weights(a_bits, a_enc)
+    Wp = [row_planes(r, w_bits, w_enc) for r in W]
+    Ap = [row_planes(r, a_bits, a_enc) for r in At]
+    w_sums = [sum(int(v) for v in r) for r in W]
+    a_sums = [sum(int(v) for v in r) for r in At]
+    return [[bitserial_dot(Wp[m], Ap[n], cw, ca, w_enc, a_enc, K, a_sums[n], w_sums[m])
+             for n in range(len(At))] for m in range(len(W))]
