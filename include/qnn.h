@@ -223,14 +223,17 @@ qnn_status qnn_im2col(const qnn_conv_desc *d, const void *in, void *lowered, voi
  * weight operand in format d->fmt.  Output: as qnn_qgemm with N = B*OH*OW,
  * M = OC, i.e. a channels-last feature map [B][OH][OW][...].  BIPOLAR
  * activations with pad > 0 are UNSUPPORTED (zero is not representable).
- * The lowered matrix of Section 3.2 is written to `workspace` only where the
- * GEMM kernel cannot form its tiles itself: bit-plane maps are lowered on the fly by the
- * staging code of the tiled AND/POPC kernel (word-granular, as in Section 3.2); 8-bit maps are lowered inside the
- * kernel (by its tensor-map loader when C and in_pitch are multiples of 16; by
- * lowering warps when pixels are contiguous and either C is not a multiple of
- * 16, pad == 0 and OC <= 128, or C is a multiple of 16 but not of 128 and the
- * layer has many tiles), with the same integer results.  The pad columns of the weight rows (see
- * qnn_conv_lowered_k) must be zero: the in-kernel lowering leaves image bytes,
+ * The lowered matrix of Section 3.2 is written to `workspace` only where the GEMM
+ * kernel cannot form its tiles itself.  Bit-plane maps are lowered on the fly by the
+ * staging code of the tiled AND/POPC kernel (word-granular, as in Section 3.2).
+ * 8-bit maps are lowered inside the tensor-core kernel: by its tensor-map loader
+ * when C and in_pitch are multiples of 16 (the CTA-pair kernel for large layers,
+ * the one-CTA kernel otherwise); by lowering warps when pixels are contiguous and
+ * either C is not a multiple of 16, pad == 0, OC <= 128 and the weights are not
+ * BIPOLAR, or C is a multiple of 16 but not of 128, the layer has many tiles and
+ * the CTA-pair kernel does not apply.  All routes give the same integer results.
+ * The pad columns of the weight rows (see qnn_conv_lowered_k) must be zero bytes
+ * for the lowering warps' unmasked route: it leaves image bytes,
  * not zeros, opposite them.  The workspace must be given in every case. */
 qnn_status qnn_qconv(const qnn_conv_desc *d, const void *Wpacked, const void *in,
                      const int32_t *thr, void *out,

@@ -875,7 +875,18 @@ struct Tc2Smem {
     int abort_flag;
 };
 
-template <int OUT_MODE, int OUT_BITS>
+// Width (MMA N) of the channel tile that starts at channel ct: 256, or what is left of M rounded up
+// to 64 (the two epilogue halves are whole 32-column chunks).
+__device__ __forceinline__ int pair_tile_width(const TcParams &p, int ct) {
+    const int left = p.M - ct;
+    return left >= T2_BN ? T2_BN : ((left + 63) & ~63);
+}
+
+// CONV: implicit convolution (see TcParams): each CTA of the pair fetches its 128 output pixels
+// through the im2col tensor map, and the last channel tile is as wide as the channels left (the
+// plain GEMM keeps 256-wide tiles and a loop body of four MMAs: the issuing thread is the one
+// thread whose instruction count shows in the kernel's time).
+template <int OUT_MODE, int OUT_BITS, bool CONV>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_constant__ CUtensorMap map_wgt,
                  const TcParams p) {
@@ -919,15 +930,33 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_const
             bool ok = true;
             for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
                 const int p0 = (tile % p.tiles_p) * 256 + (int)rank * 128;
-                const int c0 = (tile / p.tiles_p) * T2_BN + (int)rank * 128;
+                const int ct = (tile / p.tiles_p) * T2_BN;
+                // this CTA's half of the tile's channels (the copy always fetches 128 weight rows; a
+                // narrower last tile uses the first half-width of them)
+                const int c0 = ct + (int)rank * (CONV ? pair_tile_width(p, ct) >> 1 : 128);
+                int cv_w = 0, cv_h = 0, cv_n = 0;          // CONV: base pixel of this CTA's first output pixel
+                if (CONV) {
+                    cv_n = p0 / p.cv_OHW;
+                    const int r = p0 - cv_n * p.cv_OHW, oh = r / p.cv_OW;
+                    cv_h = oh * p.cv_stride - p.cv_pad;
+                    cv_w = (r - oh * p.cv_OW) * p.cv_stride - p.cv_pad;
+                }
+                int tap = 0, cc = 0, kh = 0, kw = 0;       // CONV: k-block = (filter tap, channel chunk)
                 for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
                     const int s = it % T2_STAGES;
                     const uint32_t ph = (it / T2_STAGES) & 1;
                     if (!(ok = mbar_wait(&sm.empty[s], ph ^ 1, abort_flag))) break;
                     if (rank == 0) mbar_arrive_expect_tx(&sm.full[s], PAIR_STAGE_BYTES);
                     const uint32_t leader_full = map_to_cta(smem_u32(&sm.full[s]), 0);
-                    tma_load_2d_pair(sm.act[s], &map_act, leader_full, kb * TC_BK, p0);
-                    tma_load_2d_pair(sm.wgt[s], &map_wgt, leader_full, kb * TC_BK, c0);
+                    if (CONV) {
+                        tma_load_im2col_pair(sm.act[s], &map_act, leader_full, cc * TC_BK, cv_w, cv_h, cv_n,
+                                             (uint16_t)kw, (uint16_t)kh);
+                        tma_load_2d_pair(sm.wgt[s], &map_wgt, leader_full, tap * p.cv_C + cc * TC_BK, c0);
+                        if (++cc == p.cchunks) { cc = 0; ++tap; if (++kw == p.cv_KW) { kw = 0; ++kh; } }
+                    } else {
+                        tma_load_2d_pair(sm.act[s], &map_act, leader_full, kb * TC_BK, p0);
+                        tma_load_2d_pair(sm.wgt[s], &map_wgt, leader_full, kb * TC_BK, c0);
+                    }
                 }
             }
         }
@@ -937,11 +966,17 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_const
         if (lane == 0 && rank == 0) {
             uint32_t it = 0, tcount = 0;
             bool ok = true;
+            // CONV: 32-byte slices of a tap's last channel chunk that hold real channels (4: all)
+            const int tail_c = CONV ? p.cv_C - (p.cchunks - 1) * TC_BK : TC_BK;
+            const int tail_kk = tail_c >= TC_BK ? TC_BK / 32 : (tail_c + 31) >> 5;
             for (int tile = pair; ok && tile < num_tiles; tile += num_pairs, ++tcount) {
                 const uint32_t buf = tcount & 1, acc_ph = (tcount >> 1) & 1;
                 if (!(ok = mbar_wait(&sm.tmem_empty[buf], acc_ph ^ 1, abort_flag))) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * T2_BN;
+                // MMA N: 256, or (CONV) the width of a narrower last channel tile
+                const uint32_t idesc = p.idesc | ((uint32_t)((CONV ? pair_tile_width(p, (tile / p.tiles_p) * T2_BN) : T2_BN) >> 3) << 17);
+                int cc = 0;                                // CONV: channel chunk of the k-block
                 for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
                     const int s = it % T2_STAGES;
                     const uint32_t ph = (it / T2_STAGES) & 1;
@@ -949,9 +984,16 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_const
                     tc_fence_after();
                     const uint64_t da = umma_smem_desc(smem_u32(sm.act[s]));
                     const uint64_t db = umma_smem_desc(smem_u32(sm.wgt[s]));
+                    if (CONV && tail_kk != TC_BK / 32 && cc == p.cchunks - 1) {
+                        // the last channel chunk of a tap holds fewer than 128 real bytes: skip the all-zero MMAs
+                        for (int kk = 0; kk < tail_kk; ++kk)
+                            umma_i8_pair(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (kb | kk) != 0);
+                    } else {
 #pragma unroll
-                    for (int kk = 0; kk < TC_BK / 32; ++kk)
-                        umma_i8_pair(d_tmem, da + 2 * kk, db + 2 * kk, p.idesc, (kb | kk) != 0);
+                        for (int kk = 0; kk < TC_BK / 32; ++kk)
+                            umma_i8_pair(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (kb | kk) != 0);
+                    }
+                    if (CONV && ++cc == p.cchunks) cc = 0;
                     // free the stage in both CTAs
                     umma_commit_pair(map_to_cta(smem_u32(&sm.empty[s]), 0));
                     umma_commit_pair(map_to_cta(smem_u32(&sm.empty[s]), 1));
@@ -970,7 +1012,8 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_const
                                          [&](uint32_t i, int &c0, int &bn) {
                                              const long long tile = pair + (long long)i * num_pairs;
                                              if (tile >= num_tiles) return false;
-                                             c0 = (int)(tile / p.tiles_p) * T2_BN; bn = T2_BN;
+                                             c0 = (int)(tile / p.tiles_p) * T2_BN;
+                                             bn = CONV ? pair_tile_width(p, c0) : T2_BN;
                                              return true;
                                          });
     } else {
@@ -980,8 +1023,9 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_const
             const int p0 = (tile % p.tiles_p) * 256 + (int)rank * 128, c0 = (tile / p.tiles_p) * T2_BN;
             const uint32_t buf = tcount & 1, acc_ph = (tcount >> 1) & 1;
             if (!epilogue_tile<OUT_MODE, OUT_BITS>(p, sm.thr[buf], &sm.thr_full[buf], &sm.thr_empty[buf], acc_ph,
-                                                   &sm.tmem_full[buf], acc_ph, tmem_base + buf * T2_BN, T2_BN,
-                                                   p0, c0, -1, TcExchange{}, warp, lane, abort_flag))
+                                                   &sm.tmem_full[buf], acc_ph, tmem_base + buf * T2_BN,
+                                                   CONV ? pair_tile_width(p, c0) : T2_BN, p0, c0, -1, TcExchange{}, warp,
+                                                   lane, abort_flag))
                 break;
             if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&sm.tmem_empty[buf]), 0));
         }
@@ -1114,9 +1158,9 @@ static qnn_status launch_cfg(const CUtensorMap &ma, const CUtensorMap &mw, const
     return launch_status();
 }
 
-template <int OUT_MODE, int OUT_BITS>
+template <int OUT_MODE, int OUT_BITS, bool CONV>
 static qnn_status launch_pair_cfg(const CUtensorMap &ma, const CUtensorMap &mw, const TcParams &p, cudaStream_t s) {
-    auto kern = qgemm_tc2_kernel<OUT_MODE, OUT_BITS>;
+    auto kern = qgemm_tc2_kernel<OUT_MODE, OUT_BITS, CONV>;
     const size_t smem = sizeof(Tc2Smem<OUT_BITS>) + 1024;
     static bool attr_done[QNN_MAX_DEVICES] = {false};       // per instantiation and device
     const int dev = current_device();
@@ -1165,7 +1209,7 @@ static qnn_status launch_out(int mode, int out_bits, const CUtensorMap &ma, cons
 
 static qnn_status launch_pair_out(int mode, int out_bits, const CUtensorMap &ma, const CUtensorMap &mw,
                                   const TcParams &p, cudaStream_t s) {
-#define QNN_C2(MODE_, BITS_) launch_pair_cfg<MODE_, BITS_>(ma, mw, p, s)
+#define QNN_C2(MODE_, BITS_) (p.taps ? launch_pair_cfg<MODE_, BITS_, true>(ma, mw, p, s) : launch_pair_cfg<MODE_, BITS_, false>(ma, mw, p, s))
     QNN_TC_DISPATCH(QNN_C2(OUT_RAW, 0), QNN_C2)
 #undef QNN_C2
 }
@@ -1248,7 +1292,7 @@ static qnn_status tc_launch(const qnn_gemm_desc *d, const qnn_conv_desc *cv, con
                             const int32_t *thr, void *out, cudaStream_t s) {
     const int ld = round_up(d->K, 16);
     const int sms = sm_count();
-    const bool pair = !cv && choose_pair_kernel(d, sms);
+    const bool pair = choose_pair_kernel(d, sms);
 
     TcParams p;
     p.thr = thr; p.out = out; p.M = d->M; p.N = d->N; p.K = d->K;
@@ -1276,10 +1320,16 @@ static qnn_status tc_launch(const qnn_gemm_desc *d, const qnn_conv_desc *cv, con
     CUtensorMap ma, mw;
 
     if (pair) {
-        if (!make_map(&ma, A, d->N, d->K, ld, TC_BP) || !make_map(&mw, W, d->M, d->K, ld, 128)) return QNN_ERR_CUDA;
+        if (cv) {
+            const int pitch = cv->in_pitch ? cv->in_pitch : round_up(cv->C, 16);
+            if (!make_im2col_map(&ma, A, cv, pitch)) return QNN_ERR_UNSUPPORTED;     // caller lowers explicitly
+        } else if (!make_map(&ma, A, d->N, d->K, ld, TC_BP)) {
+            return QNN_ERR_CUDA;
+        }
+        if (!make_map(&mw, W, d->M, d->K, ld, 128)) return QNN_ERR_CUDA;
         p.tiles_p = ceil_div(d->N, 256); p.tiles_c = ceil_div(d->M, T2_BN);
         p.units = p.full_units = p.tiles_p * p.tiles_c;
-        p.idesc = idesc_base | ((uint32_t)(T2_BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+        p.idesc = idesc_base | ((uint32_t)(256 >> 4) << 24);          // the kernel adds the tile's N
         return launch_pair_out(mode, d->out_bits, ma, mw, p, s);
     }
     TcPlan pl;
@@ -1368,7 +1418,11 @@ qnn_status gemm_tc_lower_launch(const qnn_conv_desc *cv, const qnn_gemm_desc *g,
         const char *force = getenv("QNN_CONV_LOWER");            // "1": skip the heuristic (tests), "0": never
         if (force && force[0] == '0') return QNN_ERR_UNSUPPORTED;
         if (cv->pad >= cv->KH || cv->pad >= cv->KW) return QNN_ERR_UNSUPPORTED;
-        if (!(force && force[0] == '1') && ((cv->C % TC_BK) == 0 || tiles < 4 * sm_count())) return QNN_ERR_UNSUPPORTED;
+        // ... and not where the CTA-pair kernel takes the convolution through the tensor-map loader
+        // (27 x 27 x 96 -> 256 at batch 256: 108 us there against 129 us here)
+        if (!(force && force[0] == '1') &&
+            ((cv->C % TC_BK) == 0 || tiles < 4 * sm_count() || choose_pair_kernel(g, sm_count())))
+            return QNN_ERR_UNSUPPORTED;
     }
 
     TcParams p;

@@ -175,6 +175,16 @@ __device__ __forceinline__ void tma_load_2d_pair(void *dst, const CUtensorMap *m
         "[%0], [%1, {%3, %4}], [%2];"
         ::"r"(smem_u32(dst)), "l"(map), "r"(bar_cluster_addr), "r"(x), "r"(y) : "memory");
 }
+// im2col-mode load of a CTA pair's kernel (see tma_load_im2col); completion bytes are counted on
+// the barrier at cluster address `bar_cluster_addr` (the pair leader's).  No multicast.
+__device__ __forceinline__ void tma_load_im2col_pair(void *dst, const CUtensorMap *map, uint32_t bar_cluster_addr,
+                                                     int c, int w, int h, int n, uint16_t woff, uint16_t hoff) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.im2col.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(bar_cluster_addr), "r"(c), "r"(w), "r"(h), "r"(n), "h"(woff), "h"(hoff)
+        : "memory");
+}
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t *dst_smem, uint32_t ncols) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)),
                  "r"(ncols) : "memory");

@@ -302,9 +302,13 @@ def test_config4_alexnet_batch256_sampled_images(qb):
     (2, 23, 17, 64, 48, 5, 3, 3, 2, 2, 2),        # stride 3 with padding, rectangular filter and image
     (4, 9, 9, 128, 130, 3, 3, 2, 1, 1, 2),        # stride 2, padding 1, a full 128-byte chunk
 ])
-def test_implicit_convolution_shapes(qb, monkeypatch, shape):
-    """Convolution with the lowering done by the tensor-core kernel's loader, against the direct
-    convolution; the explicit-lowering path must give the same bytes."""
+@pytest.mark.parametrize("kernel", ["single", "pair"])
+def test_implicit_convolution_shapes(qb, monkeypatch, shape, kernel):
+    """Convolution with the lowering done by the tensor-core kernel's loader (the one-CTA kernel
+    and the CTA-pair kernel, whose two CTAs fetch 128 output pixels each through the im2col tensor
+    map), against the direct convolution; the explicit-lowering path must give the same bytes."""
+    monkeypatch.setenv("QNN_TC_KERNEL", kernel)
+    monkeypatch.setenv("QNN_CONV_LOWER", "0")         # not the lowering warps: the tensor-map loader
     monkeypatch.setenv("QNN_CONV_IMPLICIT", "1")      # also where the library would rather lower explicitly
     case = synth.conv_case(990 + shape[3], *shape)
     x, pitch = device_map(qb, case, INT8)
