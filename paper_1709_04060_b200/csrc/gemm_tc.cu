@@ -772,6 +772,9 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
         if (lane == 0) {
             uint32_t it = 0, tcount = 0;
             bool ok = true;
+            // 32-byte slices with real data in a "tail" k-block (see below); 4: none is ever skipped
+            const int tail_bytes = p.taps ? p.cv_C - (p.cchunks - 1) * TC_BK : (LOWER ? p.K - (p.num_kb - 1) * TC_BK : TC_BK);
+            const int tail_kk = tail_bytes >= TC_BK ? TC_BK / 32 : (tail_bytes + 31) >> 5;
             if (LOWER == 1) ok = mbar_wait(&sm.w_full, 0, abort_flag);
             for (int u = blockIdx.x; ok && u < p.units; u += gridDim.x, ++tcount) {
                 const uint32_t buf = tcount & 1, acc_ph = (tcount >> 1) & 1;
@@ -780,6 +783,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
                 tc_fence_after();
                 QNN_TRACE(5, tcount);
                 const uint32_t d_tmem = tmem_base + buf * BN;
+                int cc = p.taps ? un.kb0 % p.cchunks : 0;      // implicit convolution: channel chunk of the k-block
                 for (int kb = un.kb0; kb < un.kb1; ++kb, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1;
@@ -790,20 +794,28 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
                     if (kb == un.kb0) QNN_TRACE(6, tcount);
                     const uint64_t da = umma_smem_desc(smem_u32(sm.act[s]));
                     const uint64_t db = umma_smem_desc(smem_u32(LOWER == 1 ? w_block(kb) : sm.wgt[s]));
-                    // a channel chunk may hold fewer than 128 real bytes: skip the all-zero MMAs
-                    int nk = TC_BK / 32;
-                    if (p.taps) {
-                        const int left = p.cv_C - (kb % p.cchunks) * TC_BK;
-                        if (left < TC_BK) nk = (left + 31) >> 5;
-                    }
+                    // A k-block that holds fewer than 128 real depth bytes (the last channel chunk of a
+                    // filter tap; the end of a lowered row) skips its all-zero MMAs.  Everything else
+                    // takes the loop of exactly four MMAs: this thread's instructions between MMAs are
+                    // time during which the tensor pipe may run dry.
+                    const bool tail = p.taps ? cc == p.cchunks - 1 : (LOWER != 0 && kb == p.num_kb - 1);
                     if (LOWER) {
-                        const int left = p.K - kb * TC_BK;
-                        if (left < TC_BK) nk = (left + 31) >> 5;
-                    }
+                        // (the kernels with lowering warps are bound by those warps, and measured faster
+                        // with the predicated form of the loop)
+                        const int nk = tail ? tail_kk : TC_BK / 32;
 #pragma unroll
-                    for (int kk = 0; kk < TC_BK / 32; ++kk)   // 32 depth bytes per MMA: +2 in 16-byte units
-                        if (kk < nk) umma_i8(d_tmem, da + 2 * kk, db + 2 * kk, p.idesc, (kb > un.kb0) || kk != 0);
+                        for (int kk = 0; kk < TC_BK / 32; ++kk)
+                            if (kk < nk) umma_i8(d_tmem, da + 2 * kk, db + 2 * kk, p.idesc, (kb > un.kb0) || kk != 0);
+                    } else if (tail && tail_kk != TC_BK / 32) {
+                        for (int kk = 0; kk < tail_kk; ++kk)
+                            umma_i8(d_tmem, da + 2 * kk, db + 2 * kk, p.idesc, (kb > un.kb0) || kk != 0);
+                    } else {
+#pragma unroll
+                        for (int kk = 0; kk < TC_BK / 32; ++kk)   // 32 depth bytes per MMA: +2 in 16-byte units
+                            umma_i8(d_tmem, da + 2 * kk, db + 2 * kk, p.idesc, (kb > un.kb0) || kk != 0);
+                    }
                     umma_commit(&sm.empty[s]);
+                    if (p.taps && ++cc == p.cchunks) cc = 0;
                 }
                 if (ok) umma_commit(&sm.tmem_full[buf]);
                 QNN_TRACE(7, tcount);
