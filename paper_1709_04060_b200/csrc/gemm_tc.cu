@@ -976,11 +976,18 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_const
     } else if (warp == 1) {
         // ---------------------------------------------- MMA issuer (leader CTA only)
         if (lane == 0 && rank == 0) {
-            uint32_t it = 0, tcount = 0;
+            uint32_t tcount = 0;
             bool ok = true;
             // CONV: 32-byte slices of a tap's last channel chunk that hold real channels (4: all)
             const int tail_c = CONV ? p.cv_C - (p.cchunks - 1) * TC_BK : TC_BK;
             const int tail_kk = tail_c >= TC_BK ? TC_BK / 32 : (tail_c + 31) >> 5;
+            // Everything that depends on the stage is carried incrementally (no division, no address
+            // mapping in the loop): the fewer instructions this thread runs between MMAs, the less
+            // often the tensor pipe waits for it.
+            const uint64_t da0 = umma_smem_desc(smem_u32(sm.act[0])), db0 = umma_smem_desc(smem_u32(sm.wgt[0]));
+            const uint32_t empty0 = map_to_cta(smem_u32(&sm.empty[0]), 0), empty1 = map_to_cta(smem_u32(&sm.empty[0]), 1);
+            int s = 0;                                     // stage of the ring
+            uint32_t ph = 0;                               // its phase
             for (int tile = pair; ok && tile < num_tiles; tile += num_pairs, ++tcount) {
                 const uint32_t buf = tcount & 1, acc_ph = (tcount >> 1) & 1;
                 if (!(ok = mbar_wait(&sm.tmem_empty[buf], acc_ph ^ 1, abort_flag))) break;
@@ -989,13 +996,11 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_const
                 // MMA N: 256, or (CONV) the width of a narrower last channel tile
                 const uint32_t idesc = p.idesc | ((uint32_t)((CONV ? pair_tile_width(p, (tile / p.tiles_p) * T2_BN) : T2_BN) >> 3) << 17);
                 int cc = 0;                                // CONV: channel chunk of the k-block
-                for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
-                    const int s = it % T2_STAGES;
-                    const uint32_t ph = (it / T2_STAGES) & 1;
+                for (int kb = 0; kb < p.num_kb; ++kb) {
                     if (!(ok = mbar_wait(&sm.full[s], ph, abort_flag))) break;
                     tc_fence_after();
-                    const uint64_t da = umma_smem_desc(smem_u32(sm.act[s]));
-                    const uint64_t db = umma_smem_desc(smem_u32(sm.wgt[s]));
+                    const uint64_t da = da0 + (uint64_t)(s * (TC_BP * TC_BK / 16));
+                    const uint64_t db = db0 + (uint64_t)(s * (128 * TC_BK / 16));
                     if (CONV && tail_kk != TC_BK / 32 && cc == p.cchunks - 1) {
                         // the last channel chunk of a tap holds fewer than 128 real bytes: skip the all-zero MMAs
                         for (int kk = 0; kk < tail_kk; ++kk)
@@ -1007,8 +1012,9 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_const
                     }
                     if (CONV && ++cc == p.cchunks) cc = 0;
                     // free the stage in both CTAs
-                    umma_commit_pair(map_to_cta(smem_u32(&sm.empty[s]), 0));
-                    umma_commit_pair(map_to_cta(smem_u32(&sm.empty[s]), 1));
+                    umma_commit_pair(empty0 + 8u * (uint32_t)s);
+                    umma_commit_pair(empty1 + 8u * (uint32_t)s);
+                    if (++s == T2_STAGES) { s = 0; ph ^= 1u; }
                 }
                 if (ok) {
                     umma_commit_pair(map_to_cta(smem_u32(&sm.tmem_full[buf]), 0));
