@@ -133,7 +133,18 @@ typedef struct {
                              operand counts as one plane (index 0).               */
 } qnn_gemm_desc;
 
-/* Scratch bytes qnn_qgemm needs for this problem (may be 0).  Host only. */
+/* Scratch bytes qnn_qgemm can use for this problem (0: none).  The workspace is OPTIONAL:
+ * without it (NULL, or fewer bytes) the call computes the same result.  With it, the CTA-pair
+ * tensor-core kernel splits a last round of 256 x 256 tiles that would keep at most half of the
+ * SM pairs busy: two neighbouring pairs take one half of the depth each and exchange int32
+ * partial sums through the workspace (Section 4.1 of the paper measures exactly such large square
+ * products; the split is worth 2-4 % there).  Contract: 16-byte aligned; its first 8192 bytes
+ * are flag words that must be ZERO before the first call that uses the workspace; the kernel
+ * leaves them zero, so the same workspace serves call after call (after a call that ended in
+ * QNN_ERR_DEVICE_TIMEOUT, zero them again).  Calls that may run concurrently (different streams)
+ * need different workspaces, and a call that uses one should have the GPU's SMs to itself apart
+ * from kernels that do not wait on others: the two pairs of a split tile wait for each other (a
+ * bounded wait, ending in QNN_ERR_DEVICE_TIMEOUT).  Host only. */
 size_t qnn_gemm_workspace_bytes(const qnn_gemm_desc *d);
 
 /* Bytes of the output buffer for this problem (see qnn_qgemm).  Host only. */

@@ -321,8 +321,9 @@ def qgemm(d: qnn_gemm_desc, W, A, thr, out=None, stream=None) -> torch.Tensor:
     [N][M] when thr is None)."""
     if out is None:
         out = _dev_bytes(qnn_gemm_out_bytes(d, thr is not None))
+    # the optional workspace starts with flag words that must be zero before the first call
     ws_bytes = qnn_gemm_workspace_bytes(d)
-    ws = _dev_bytes(ws_bytes) if ws_bytes else None
+    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device="cuda") if ws_bytes else None
     check(qnn_qgemm(d, W, A, thr, out, ws, ws_bytes, stream))
     if thr is None:
         return out[: d.N * d.M * 4].view(torch.int32).view(d.N, d.M)

@@ -148,8 +148,11 @@ qnn_status qnn_pack(const qnn_pack_desc *d, const void *logical, void *packed, v
 }
 
 size_t qnn_gemm_workspace_bytes(const qnn_gemm_desc *d) {
-    (void)d;
-    return 0;
+    int path = 0;
+    if (check_gemm_desc(d, true, &path) != QNN_OK) return 0;
+    if (d->w_fmt != QNN_FMT_INT8 || path != QNN_PATH_TCGEN05_I8) return 0;
+    if (d->path == QNN_PATH_AUTO && gemv_i8_fits(d)) return 0;
+    return gemm_tc_workspace_bytes(d);
 }
 
 size_t qnn_gemm_out_bytes(const qnn_gemm_desc *d, int has_thresholds) {
@@ -173,7 +176,6 @@ int qnn_qgemm_kernel(const qnn_gemm_desc *d, int has_thresholds) {
 
 qnn_status qnn_qgemm(const qnn_gemm_desc *d, const void *W, const void *A, const int32_t *thr,
                      void *out, void *workspace, size_t workspace_bytes, void *stream) {
-    (void)workspace; (void)workspace_bytes;
     int path = 0;
     qnn_status st = check_gemm_desc(d, thr != nullptr, &path);
     if (st != QNN_OK) return st;
@@ -185,7 +187,12 @@ qnn_status qnn_qgemm(const qnn_gemm_desc *d, const void *W, const void *A, const
     // one warp per weight row (a tensor-core tile would be almost empty)
     if (d->path == QNN_PATH_AUTO && d->w_fmt == QNN_FMT_INT8 && gemv_i8_fits(d))
         return gemv_i8_launch(d, W, A, thr, out, (cudaStream_t)stream);
-    if (path == QNN_PATH_TCGEN05_I8) return gemm_tc_launch(d, W, A, thr, out, (cudaStream_t)stream);
+    if (path == QNN_PATH_TCGEN05_I8) {
+        // the workspace is optional (see the header): used only when given, large enough and aligned
+        const bool ws_ok = workspace && aligned16(workspace);
+        return gemm_tc_launch(d, W, A, thr, out, ws_ok ? workspace : nullptr, ws_ok ? workspace_bytes : 0,
+                              (cudaStream_t)stream);
+    }
     // a handful of columns: stream the weight planes once, one warp per row
     if (gemv_planes_fits(d)) return gemv_planes_launch(d, W, A, thr, out, (cudaStream_t)stream);
     return gemm_bitserial_launch(d, W, A, thr, out, (cudaStream_t)stream);

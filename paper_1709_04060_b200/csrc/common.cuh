@@ -75,7 +75,8 @@ bool gemv_fields_fits(const qnn_gemm_desc *d, bool has_thr);
 qnn_status gemv_fields_launch(const qnn_gemm_desc *d, const void *W, const void *A,
                               const int32_t *thr, void *out, cudaStream_t s);
 qnn_status gemm_tc_launch(const qnn_gemm_desc *d, const void *W, const void *A,
-                          const int32_t *thr, void *out, cudaStream_t s);
+                          const int32_t *thr, void *out, void *ws, size_t ws_bytes, cudaStream_t s);
+size_t gemm_tc_workspace_bytes(const qnn_gemm_desc *d);   // optional scratch of the CTA-pair kernel (0: none)
 bool gemm_tc_uses_pair_kernel(const qnn_gemm_desc *d);
 qnn_status gemm_tc_conv_launch(const qnn_conv_desc *cv, const qnn_gemm_desc *g, const void *W, const void *in,
                                const int32_t *thr, void *out, cudaStream_t s);

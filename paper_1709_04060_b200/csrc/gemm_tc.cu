@@ -109,6 +109,12 @@ struct TcParams {
     int lw_step;           // stride*C: bytes between the runs of neighbouring output pixels
     int lw_run, lw_vecs;   // bytes of a run (KW*C) and its 16-byte pieces
     int lw_stage_bytes;    // bytes of one staging buffer
+    // CTA-pair kernel with a split last round (see qgemm_tc2_kernel): the depth of each of the last
+    // split_rem tiles is shared by two neighbouring CTA pairs, which exchange int32 partial sums
+    // through global memory.
+    int split_rem;             // tiles of the last round (0: nothing is split)
+    unsigned *split_flags;     // [split_rem][part][rank][epilogue warp]: 1 = that warp's partial sums are in its slab
+    int4 *split_slabs;         // same index: 2 chunks x 32 lanes x 32 columns of int32
 };
 
 constexpr int LW_WARPS = 4;                    // lowering warps of the LOWER kernels
@@ -871,6 +877,10 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_consta
 // leader's mbarrier.
 constexpr int T2_STAGES = 6;
 constexpr int T2_BN = 256;
+enum { PAIR_PLAIN = 0, PAIR_CONV = 1, PAIR_SPLIT = 2 };
+constexpr int SPLIT_FLAG_BYTES = 8192;                   // flags of the split last round, at the start of the workspace
+constexpr int SPLIT_SLAB_INT4 = 2 * 8 * 32;              // one epilogue warp's partial sums: 2 chunks of 32 x 32 int32
+constexpr size_t SPLIT_TILE_BYTES = (size_t)2 * 2 * EPI_WARPS * SPLIT_SLAB_INT4 * 16;   // both parts, both CTAs: 256 KB
 
 template <int OUT_BITS>
 struct Tc2Smem {
@@ -894,14 +904,129 @@ __device__ __forceinline__ int pair_tile_width(const TcParams &p, int ct) {
     return left >= T2_BN ? T2_BN : ((left + 63) & ~63);
 }
 
-// CONV: implicit convolution (see TcParams): each CTA of the pair fetches its 128 output pixels
-// through the im2col tensor map, and the last channel tile is as wide as the channels left (the
-// plain GEMM keeps 256-wide tiles and a loop body of four MMAs: the issuing thread is the one
+// One unit of work of a CTA pair: a whole tile, or (PAIR_SPLIT, last round) one half of a tile's depth.
+struct PairUnit { int tile, kb_lo, kb_hi, part, j; };      // part < 0: whole tile; else j = index among the split tiles
+template <int KIND>
+__device__ __forceinline__ PairUnit pair_unit(const TcParams &p, int u, int num_tiles) {
+    PairUnit r;
+    r.tile = u; r.kb_lo = 0; r.kb_hi = p.num_kb; r.part = -1; r.j = 0;
+    if (KIND == PAIR_SPLIT) {
+        const int full = num_tiles - p.split_rem;
+        if (u >= full) {
+            r.j = (u - full) >> 1; r.part = (u - full) & 1;
+            r.tile = full + r.j;
+            r.kb_lo = r.part ? p.num_kb >> 1 : 0;
+            r.kb_hi = r.part ? p.num_kb : p.num_kb >> 1;
+        }
+    }
+    return r;
+}
+
+// Epilogue of a split unit.  The pair that ran depth part `part` of tile j finishes the 64-column
+// groups g with (g & 1) == part and sends its partial sums of the other groups to the pair that ran
+// the other part (the neighbouring pair, busy with the same tile at the same time).  Every epilogue
+// warp covers two groups: it first writes the one it does not own to its slab in global memory and
+// raises its flag (release), then waits (bounded) for the flag of the same warp of the partner pair,
+// adds the partner's slab to the group it owns, counts thresholds and stores.  The reader clears the
+// flag, so the flags are zero again when the kernel ends.
+template <int OUT_MODE, int OUT_BITS>
+__device__ __forceinline__ bool epilogue_tile_split(const TcParams &p, const int *thr_s, uint64_t *thr_full,
+                                                    uint64_t *thr_empty, uint32_t thr_parity, uint64_t *tmem_full,
+                                                    uint32_t full_parity, uint32_t t_acc, int p0, int c0,
+                                                    const PairUnit &un, uint32_t rank, int warp, int lane,
+                                                    volatile int *abort_flag) {
+    constexpr int NT = thr_slots(OUT_BITS);
+    const int quad = warp & 3, half = (warp - 2) >> 2, ew = warp - 2;
+    if (OUT_MODE != OUT_RAW && !warp_wait(thr_full, thr_parity, lane, abort_flag)) return false;
+    if (!warp_wait(tmem_full, full_parity, lane, abort_flag)) return false;
+    tc_fence_after();
+    const uint32_t t_row = t_acc + ((uint32_t)(quad * 32) << 16);
+    const int n = p0 + quad * 32 + lane;
+    const int own_c = half * 128 + un.part * 64, send_c = half * 128 + (un.part ^ 1) * 64;
+    const size_t mine = (size_t)((un.j * 2 + un.part) * 2 + (int)rank) * EPI_WARPS + ew;
+    const size_t theirs = (size_t)((un.j * 2 + (un.part ^ 1)) * 2 + (int)rank) * EPI_WARPS + ew;
+    int acc[32];
+    // ---- send (chunks wholly beyond M are neither sent nor awaited: both sides skip them alike)
+    {
+        int4 *slab = p.split_slabs + mine * SPLIT_SLAB_INT4;
+#pragma unroll 1
+        for (int c = 0; c < 2; ++c) {
+            if (c0 + send_c + 32 * c >= p.M) break;
+            tmem_ld32_issue(t_row + send_c + 32 * c, acc);
+            tmem_ld_wait(acc);
+#pragma unroll
+            for (int v = 0; v < 8; ++v)
+                slab[(c * 8 + v) * 32 + lane] = make_int4(acc[4 * v], acc[4 * v + 1], acc[4 * v + 2], acc[4 * v + 3]);
+        }
+        __syncwarp();
+        // the warp's stores happen before lane 0's release (ordered by the __syncwarp above, made
+        // visible GPU-wide by the release); a group wholly beyond M has no reader
+        if (lane == 0 && c0 + send_c < p.M)
+            asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.split_flags + mine), "r"(1u) : "memory");
+    }
+    // ---- receive, add, finish
+    bool ok = true;
+    if (c0 + own_c < p.M) {
+        if (lane == 0) {
+            const unsigned *flag = p.split_flags + theirs;
+            const long long t0 = clock64();
+            for (;;) {
+                unsigned v;
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+                if (v != 0u) break;
+                if (*abort_flag) { ok = false; break; }
+                if (clock64() - t0 > TC_WAIT_CYCLES) {
+                    *abort_flag = 1;
+                    atomicExch(&g_dev_status, (int)QNN_ERR_DEVICE_TIMEOUT);
+                    ok = false;
+                    break;
+                }
+                __nanosleep(100);
+            }
+        }
+        ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+        if (!ok) return false;
+        const int4 *slab = p.split_slabs + theirs * SPLIT_SLAB_INT4;
+        // both chunks' partial sums are requested before the first is used (one L2 round trip, not two)
+        int4 q[2][8];
+#pragma unroll
+        for (int c = 0; c < 2; ++c)
+#pragma unroll
+            for (int v = 0; v < 8; ++v) q[c][v] = __ldcg(slab + (c * 8 + v) * 32 + lane);
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+            if (c0 + own_c + 32 * c >= p.M) break;
+            tmem_ld32_issue(t_row + own_c + 32 * c, acc);
+            tmem_ld_wait(acc);
+#pragma unroll
+            for (int v = 0; v < 8; ++v) {
+                acc[4 * v] += q[c][v].x; acc[4 * v + 1] += q[c][v].y; acc[4 * v + 2] += q[c][v].z; acc[4 * v + 3] += q[c][v].w;
+            }
+            epilogue_chunk<OUT_MODE, OUT_BITS>(p, thr_s + (own_c + 32 * c) * NT, acc, n, n < p.N, c0 + own_c + 32 * c);
+        }
+        __syncwarp();
+        if (lane == 0) *(volatile unsigned *)(p.split_flags + theirs) = 0u;     // consumed: zero for the next launch
+    }
+    tc_fence_before();
+    __syncwarp();
+    if (OUT_MODE != OUT_RAW && lane == 0) mbar_arrive(thr_empty);
+    return true;
+}
+
+// KIND PAIR_CONV: implicit convolution (see TcParams): each CTA of the pair fetches its 128 output
+// pixels through the im2col tensor map, and the last channel tile is as wide as the channels left
+// (the plain GEMM keeps 256-wide tiles and a loop body of four MMAs: the issuing thread is the one
 // thread whose instruction count shows in the kernel's time).
-template <int OUT_MODE, int OUT_BITS, bool CONV>
+// KIND PAIR_SPLIT: a plain GEMM whose last round of tiles would leave at least half of the pairs
+// idle: each of those tiles is run by two neighbouring pairs, one per half of the depth, which
+// exchange partial sums through the caller's workspace (epilogue_tile_split).  All CTAs of the
+// grid are resident together (one per SM), and the partner works on the same tile at the same
+// time, so the bounded wait normally lasts a few hundred cycles.
+template <int OUT_MODE, int OUT_BITS, int KIND>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_constant__ CUtensorMap map_wgt,
                  const TcParams p) {
+    constexpr bool CONV = KIND == PAIR_CONV;
     extern __shared__ uint8_t smem_raw[];
     using Smem = Tc2Smem<OUT_BITS>;
     // 1024-byte alignment by an offset into the array (not by rounding the pointer's integer
@@ -934,13 +1059,16 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_const
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint32_t tmem_base = sm.tmem_base;
     const int num_tiles = p.tiles_p * p.tiles_c;       // tiles of 256 pixels x 256 channels
+    const int num_units = num_tiles + (KIND == PAIR_SPLIT ? p.split_rem : 0);
 
     if (warp == 0) {
         // ---------------------------------------- producer (one per CTA, own halves)
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+            for (int u = pair; ok && u < num_units; u += num_pairs) {
+                const PairUnit un = pair_unit<KIND>(p, u, num_tiles);
+                const int tile = un.tile;
                 const int p0 = (tile % p.tiles_p) * 256 + (int)rank * 128;
                 const int ct = (tile / p.tiles_p) * T2_BN;
                 // this CTA's half of the tile's channels (the copy always fetches 128 weight rows; a
@@ -954,7 +1082,7 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_const
                     cv_w = (r - oh * p.cv_OW) * p.cv_stride - p.cv_pad;
                 }
                 int tap = 0, cc = 0, kh = 0, kw = 0;       // CONV: k-block = (filter tap, channel chunk)
-                for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
+                for (int kb = un.kb_lo; kb < un.kb_hi; ++kb, ++it) {
                     const int s = it % T2_STAGES;
                     const uint32_t ph = (it / T2_STAGES) & 1;
                     if (!(ok = mbar_wait(&sm.empty[s], ph ^ 1, abort_flag))) break;
@@ -988,7 +1116,10 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_const
             const uint32_t empty0 = map_to_cta(smem_u32(&sm.empty[0]), 0), empty1 = map_to_cta(smem_u32(&sm.empty[0]), 1);
             int s = 0;                                     // stage of the ring
             uint32_t ph = 0;                               // its phase
-            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs, ++tcount) {
+            for (int u = pair; ok && u < num_units; u += num_pairs, ++tcount) {
+                const PairUnit un = pair_unit<KIND>(p, u, num_tiles);
+                const int tile = un.tile;
+                const int unit_kb = un.kb_hi - un.kb_lo;   // all k-blocks, or (a split tile) one half of them
                 const uint32_t buf = tcount & 1, acc_ph = (tcount >> 1) & 1;
                 if (!(ok = mbar_wait(&sm.tmem_empty[buf], acc_ph ^ 1, abort_flag))) break;
                 tc_fence_after();
@@ -996,7 +1127,7 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_const
                 // MMA N: 256, or (CONV) the width of a narrower last channel tile
                 const uint32_t idesc = p.idesc | ((uint32_t)((CONV ? pair_tile_width(p, (tile / p.tiles_p) * T2_BN) : T2_BN) >> 3) << 17);
                 int cc = 0;                                // CONV: channel chunk of the k-block
-                for (int kb = 0; kb < p.num_kb; ++kb) {
+                for (int kb = 0; kb < unit_kb; ++kb) {
                     if (!(ok = mbar_wait(&sm.full[s], ph, abort_flag))) break;
                     tc_fence_after();
                     const uint64_t da = da0 + (uint64_t)(s * (TC_BP * TC_BK / 16));
@@ -1028,22 +1159,30 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_const
         if (OUT_MODE != OUT_RAW)
             stager_loop<OUT_BITS, T2_BN>(p, &sm.thr[0][0], sm.thr_full, sm.thr_empty, lane, abort_flag,
                                          [&](uint32_t i, int &c0, int &bn) {
-                                             const long long tile = pair + (long long)i * num_pairs;
-                                             if (tile >= num_tiles) return false;
-                                             c0 = (int)(tile / p.tiles_p) * T2_BN;
+                                             const long long u = pair + (long long)i * num_pairs;
+                                             if (u >= num_units) return false;
+                                             const int tile = pair_unit<KIND>(p, (int)u, num_tiles).tile;
+                                             c0 = (tile / p.tiles_p) * T2_BN;
                                              bn = CONV ? pair_tile_width(p, c0) : T2_BN;
                                              return true;
                                          });
     } else {
         // ----------------------------- epilogue (each CTA: its 128 pixels, all 256 channels)
         uint32_t tcount = 0;
-        for (int tile = pair; tile < num_tiles; tile += num_pairs, ++tcount) {
+        for (int u = pair; u < num_units; u += num_pairs, ++tcount) {
+            const PairUnit un = pair_unit<KIND>(p, u, num_tiles);
+            const int tile = un.tile;
             const int p0 = (tile % p.tiles_p) * 256 + (int)rank * 128, c0 = (tile / p.tiles_p) * T2_BN;
             const uint32_t buf = tcount & 1, acc_ph = (tcount >> 1) & 1;
-            if (!epilogue_tile<OUT_MODE, OUT_BITS>(p, sm.thr[buf], &sm.thr_full[buf], &sm.thr_empty[buf], acc_ph,
-                                                   &sm.tmem_full[buf], acc_ph, tmem_base + buf * T2_BN,
-                                                   CONV ? pair_tile_width(p, c0) : T2_BN, p0, c0, -1, TcExchange{}, warp,
-                                                   lane, abort_flag))
+            if (KIND == PAIR_SPLIT && un.part >= 0) {
+                if (!epilogue_tile_split<OUT_MODE, OUT_BITS>(p, sm.thr[buf], &sm.thr_full[buf], &sm.thr_empty[buf], acc_ph,
+                                                             &sm.tmem_full[buf], acc_ph, tmem_base + buf * T2_BN, p0, c0, un,
+                                                             rank, warp, lane, abort_flag))
+                    break;
+            } else if (!epilogue_tile<OUT_MODE, OUT_BITS>(p, sm.thr[buf], &sm.thr_full[buf], &sm.thr_empty[buf], acc_ph,
+                                                          &sm.tmem_full[buf], acc_ph, tmem_base + buf * T2_BN,
+                                                          CONV ? pair_tile_width(p, c0) : T2_BN, p0, c0, -1, TcExchange{}, warp,
+                                                          lane, abort_flag))
                 break;
             if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&sm.tmem_empty[buf]), 0));
         }
@@ -1176,9 +1315,9 @@ static qnn_status launch_cfg(const CUtensorMap &ma, const CUtensorMap &mw, const
     return launch_status();
 }
 
-template <int OUT_MODE, int OUT_BITS, bool CONV>
+template <int OUT_MODE, int OUT_BITS, int KIND>
 static qnn_status launch_pair_cfg(const CUtensorMap &ma, const CUtensorMap &mw, const TcParams &p, cudaStream_t s) {
-    auto kern = qgemm_tc2_kernel<OUT_MODE, OUT_BITS, CONV>;
+    auto kern = qgemm_tc2_kernel<OUT_MODE, OUT_BITS, KIND>;
     const size_t smem = sizeof(Tc2Smem<OUT_BITS>) + 1024;
     static bool attr_done[QNN_MAX_DEVICES] = {false};       // per instantiation and device
     const int dev = current_device();
@@ -1227,7 +1366,9 @@ static qnn_status launch_out(int mode, int out_bits, const CUtensorMap &ma, cons
 
 static qnn_status launch_pair_out(int mode, int out_bits, const CUtensorMap &ma, const CUtensorMap &mw,
                                   const TcParams &p, cudaStream_t s) {
-#define QNN_C2(MODE_, BITS_) (p.taps ? launch_pair_cfg<MODE_, BITS_, true>(ma, mw, p, s) : launch_pair_cfg<MODE_, BITS_, false>(ma, mw, p, s))
+#define QNN_C2(MODE_, BITS_) (p.taps ? launch_pair_cfg<MODE_, BITS_, PAIR_CONV>(ma, mw, p, s)                      \
+                                     : (p.split_rem ? launch_pair_cfg<MODE_, BITS_, PAIR_SPLIT>(ma, mw, p, s)     \
+                                                    : launch_pair_cfg<MODE_, BITS_, PAIR_PLAIN>(ma, mw, p, s)))
     QNN_TC_DISPATCH(QNN_C2(OUT_RAW, 0), QNN_C2)
 #undef QNN_C2
 }
@@ -1305,9 +1446,26 @@ static bool tc_plan(const qnn_gemm_desc *d, int sms, int num_kb, TcPlan *pl) {
 
 bool gemm_tc_uses_pair_kernel(const qnn_gemm_desc *d) { return choose_pair_kernel(d, sm_count()); }
 
+// Split last round of the CTA-pair kernel: the number of tiles whose depth two pairs share (0: no
+// split).  Applies when the tiles fill whole rounds of all pairs plus a last round that would keep
+// at most half of the pairs busy, and the depth has at least two k-blocks.
+static int pair_split_tiles(const qnn_gemm_desc *d, int sms) {
+    if (!choose_pair_kernel(d, sms)) return 0;
+    const long long tiles = (long long)ceil_div(d->N, 256) * ceil_div(d->M, T2_BN);
+    const int pairs = sms / 2;
+    if (pairs < 2 || tiles < pairs || ceil_div(d->K, TC_BK) < 2) return 0;
+    const int rem = (int)(tiles % pairs);
+    return (rem > 0 && 2 * rem <= pairs) ? rem : 0;
+}
+
+size_t gemm_tc_workspace_bytes(const qnn_gemm_desc *d) {
+    const int rem = pair_split_tiles(d, sm_count());
+    return rem ? (size_t)SPLIT_FLAG_BYTES + (size_t)rem * SPLIT_TILE_BYTES : 0;
+}
+
 // cv != nullptr: implicit convolution, A is the feature map (see TcParams); d is the lowered GEMM.
 static qnn_status tc_launch(const qnn_gemm_desc *d, const qnn_conv_desc *cv, const void *W, const void *A,
-                            const int32_t *thr, void *out, cudaStream_t s) {
+                            const int32_t *thr, void *out, void *ws, size_t ws_bytes, cudaStream_t s) {
     const int ld = round_up(d->K, 16);
     const int sms = sm_count();
     const bool pair = choose_pair_kernel(d, sms);
@@ -1317,6 +1475,7 @@ static qnn_status tc_launch(const qnn_gemm_desc *d, const qnn_conv_desc *cv, con
     p.num_kb = ceil_div(d->K, TC_BK);
     p.ld_out = round_up(d->M, 16);
     p.kb_half = 0; p.share = 0;
+    p.split_rem = 0; p.split_flags = nullptr; p.split_slabs = nullptr;
     p.taps = 0; p.cchunks = 1; p.cv_C = p.cv_KW = p.cv_OW = p.cv_OHW = p.cv_stride = 1; p.cv_pad = 0;
     if (cv) {
         p.taps = cv->KH * cv->KW; p.cchunks = ceil_div(cv->C, TC_BK);
@@ -1348,6 +1507,14 @@ static qnn_status tc_launch(const qnn_gemm_desc *d, const qnn_conv_desc *cv, con
         p.tiles_p = ceil_div(d->N, 256); p.tiles_c = ceil_div(d->M, T2_BN);
         p.units = p.full_units = p.tiles_p * p.tiles_c;
         p.idesc = idesc_base | ((uint32_t)(256 >> 4) << 24);          // the kernel adds the tile's N
+        // a workspace from the caller lets the last, at most half-filled round be split between pairs
+        const int rem = cv ? 0 : pair_split_tiles(d, sms);
+        if (rem && ws && ws_bytes >= (size_t)SPLIT_FLAG_BYTES + (size_t)rem * SPLIT_TILE_BYTES &&
+            (size_t)rem * 2 * 2 * EPI_WARPS * sizeof(unsigned) <= (size_t)SPLIT_FLAG_BYTES) {
+            p.split_rem = rem;
+            p.split_flags = reinterpret_cast<unsigned *>(ws);
+            p.split_slabs = reinterpret_cast<int4 *>(reinterpret_cast<uint8_t *>(ws) + SPLIT_FLAG_BYTES);
+        }
         return launch_pair_out(mode, d->out_bits, ma, mw, p, s);
     }
     TcPlan pl;
@@ -1378,8 +1545,8 @@ static qnn_status tc_launch(const qnn_gemm_desc *d, const qnn_conv_desc *cv, con
 }
 
 qnn_status gemm_tc_launch(const qnn_gemm_desc *d, const void *W, const void *A, const int32_t *thr,
-                          void *out, cudaStream_t s) {
-    return tc_launch(d, nullptr, W, A, thr, out, s);
+                          void *out, void *ws, size_t ws_bytes, cudaStream_t s) {
+    return tc_launch(d, nullptr, W, A, thr, out, ws, ws_bytes, s);
 }
 
 // Convolution without a lowered matrix: the GEMM's loader reads the 8-bit channels-last map
@@ -1400,7 +1567,7 @@ qnn_status gemm_tc_conv_launch(const qnn_conv_desc *cv, const qnn_gemm_desc *g, 
     if (!(force && force[0] == '1') && tiles <= sm_count() &&
         cv->KH * cv->KW * ceil_div(cv->C, TC_BK) > ceil_div(g->K, TC_BK))
         return QNN_ERR_UNSUPPORTED;
-    return tc_launch(g, cv, W, in, thr, out, s);
+    return tc_launch(g, cv, W, in, thr, out, nullptr, 0, s);
 }
 
 // Convolution of an 8-bit map with contiguous pixels, lowered inside the kernel (see TcParams).

@@ -190,6 +190,48 @@ def test_partial_last_round_is_shared_by_cta_pairs(qb, monkeypatch, M, N, K, w, 
     assert torch.equal(shared, whole)
 
 
+@pytest.mark.parametrize("M,N,K,w,a", [
+    (512, 11520, 512, 1, 2),     # 90 tiles on 74 SM pairs: the last 16 are split, 2 + 2 k-blocks
+    (480, 11520, 384, 2, 3),     # ragged last channel tile (224 of 256), 1 + 2 k-blocks, bisection epilogue
+    (320, 12800, 700, 4, 4),     # second channel tile holds 64 channels: three column groups have no owner
+    (768, 8448, 272, 1, 1),      # 99 tiles: 25 split, the second half of the depth is a ragged k-block
+])
+def test_pair_kernel_split_last_round(qb, monkeypatch, M, N, K, w, a):
+    """CTA-pair kernel with a workspace: the tiles of a last round that would keep at most half of the
+    SM pairs busy are each run by two neighbouring pairs, one per half of the depth, which exchange
+    int32 partial sums through the workspace.  Every output against the oracle, every output mode;
+    the same bytes as without a workspace; the workspace's flag words are zero again afterwards, so
+    that a second call on the same workspace works."""
+    monkeypatch.setenv("QNN_TC_KERNEL", "pair")
+    case = synth.gemm_case(1300 + M + K, M, N, K, w, a)
+    d = qb.gemm_desc(M, N, K, w, a, case.out_bits, case.w_enc, case.a_enc, INT8, INT8)
+    ws_bytes = qb.qnn_gemm_workspace_bytes(d)
+    if torch.cuda.get_device_properties(0).multi_processor_count == 148:
+        assert ws_bytes > 0
+    if ws_bytes == 0:
+        pytest.skip("this GPU's SM count gives the shape no half-empty last round")
+    run_case(qb, case, INT8, INT8)
+    run_case(qb, case, INT8, BITPLANES)
+    run_case(qb, case, INT8, INT8, raw=True)
+    Wp = qb.pack(qb.to_device_logical(case.W, case.w_enc), w, case.w_enc, INT8)
+    Ap = qb.pack(qb.to_device_logical(case.At, case.a_enc), a, case.a_enc, INT8)
+    thr = torch.from_numpy(case.thr).cuda()
+    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device="cuda")
+    outs = []
+    for _ in range(3):                              # the same workspace three times in a row
+        out = torch.empty(qb.qnn_gemm_out_bytes(d, True), dtype=torch.uint8, device="cuda")
+        qb.check(qb.qnn_qgemm(d, Wp, Ap, thr, out, ws, ws_bytes))
+        outs.append(out)
+    whole = torch.empty_like(outs[0])
+    qb.check(qb.qnn_qgemm(d, Wp, Ap, thr, whole, None, 0))       # no workspace: nothing is split
+    torch.cuda.synchronize()
+    st, dev = qb.qnn_device_status()
+    assert st == 0 and dev == 0
+    for out in outs:
+        assert torch.equal(out, whole)
+    assert int(ws[:8192].view(torch.int32).abs().sum()) == 0
+
+
 @pytest.mark.parametrize("which", ["single", "pair"])
 def test_integer_count_path_for_large_accumulators(qb, force_tc_kernel, which):
     """8-bit x 8-bit with K large enough that |acc| can exceed 2^24: the epilogue must
@@ -243,6 +285,11 @@ def test_full_size_4096_sampled(qb, w, a):
     for q in range(case.thr.shape[1]):
         recount += raw >= case.thr[None, :, q]
     assert np.array_equal(codes, recount)
+    # qb.qgemm hands the library its optional workspace (a split last round of tiles on GPUs whose
+    # SM count leaves one); the same call without a workspace must give the same bytes
+    whole = torch.empty(qb.qnn_gemm_out_bytes(d, True), dtype=torch.uint8, device="cuda")
+    qb.check(qb.qnn_qgemm(d, Wp, Ap, thr, whole, None, 0))
+    assert np.array_equal(whole.cpu().numpy().reshape(4096, 4096), codes)
     dp = qb.gemm_desc(4096, 4096, 4096, w, a, a, case.w_enc, case.a_enc, INT8, BITPLANES)
     planes = qb.qgemm(dp, Wp, Ap, thr).cpu().numpy()
     assert np.array_equal(decode_out(planes, BITPLANES, a, 4096, 4096, False), codes.astype(np.int64))

@@ -6,6 +6,7 @@ import os
 import re
 
 import pytest
+import torch
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
@@ -145,6 +146,26 @@ def test_argument_validation_without_launch(qb):
 
     pl = qb.qnn_pool_desc(1, 2, 2, 16, 3, 2, 2, 1)
     assert qb.qnn_maxpool(pl, P, P, stream=0) == qb.QNN_ERR_INVALID_ARG
+
+
+def test_gemm_workspace_size_rule(qb):
+    """qnn_gemm_workspace_bytes (host only; 148 SMs assumed when there is no GPU): non-zero exactly
+    where the CTA-pair kernel would leave a last round of tiles at most half full -- 8192 bytes of
+    flags plus 256 KB per tile of that round."""
+    if torch.cuda.is_available() and torch.cuda.get_device_properties(0).multi_processor_count != 148:
+        pytest.skip("the expected sizes are those of 74 SM pairs")
+    I8, PL = qb.QNN_FMT_INT8, qb.QNN_FMT_BITPLANES
+
+    def ws(M, N, K, fmt=I8):
+        return qb.qnn_gemm_workspace_bytes(qb.qnn_gemm_desc(M, N, K, 1, 2, 2, 2, 0, fmt, fmt, I8, 0, 0))
+
+    assert ws(4096, 4096, 4096) == 8192 + 34 * 256 * 1024     # 256 tiles on 74 pairs: 3 rounds + 34
+    assert ws(5120, 5120, 5120) == 8192 + 30 * 256 * 1024     # 400 tiles: 5 rounds + 30
+    assert ws(8192, 8192, 8192) == 0                          # 1024 tiles: the last round holds 62 of 74
+    assert ws(4096, 4096, 128) == 0                           # one k-block: nothing to split
+    assert ws(4096, 1024, 4096) == 0                          # not the CTA-pair kernel
+    assert ws(64, 256, 576) == 0
+    assert ws(4096, 4096, 4096, PL) == 0                      # bit planes: another path
 
 
 def test_kernel_choice_follows_the_documented_rule(qb):
