@@ -35,6 +35,8 @@
  *   QNN_CONV_IMPLICIT=1        qnn_qconv lowers inside the GEMM wherever it can
  *   QNN_CONV_LOWER=1|0         qnn_qconv uses the aligned lowering warps wherever they
  *                              apply | never
+ *   QNN_FIELDS_KERNEL=dp4a|tensor  packed (FIELDS) weights: byte dot products on the CUDA
+ *                              cores for up to 16 columns | always the tensor-core form
  *
  * Operand formats
  *   QNN_FMT_BITPLANES  uint32 [bits][rows][kw], kw = ceil(K/32): plane i holds
@@ -178,7 +180,10 @@ qnn_status qnn_qgemm(const qnn_gemm_desc *d, const void *W, const void *A,
  *                       tensor-core kernel
  *   BITPLANES operands  N <= 16: one warp per weight row over the planes; else the tiled
  *                       AND/POPC kernel
- *   FIELDS weights      N <= 16 only: packed weights expanded inside the tensor-core kernel
+ *   FIELDS weights      N <= 16 only: one column (two with 1- or 2-bit fields): one warp per
+ *                       packed weight row, an AND and a 4-way byte dot product per word and
+ *                       field position; more columns: packed weights expanded inside a
+ *                       tensor-core kernel
  * Returns a qnn_kernel value, or the (negative) qnn_status qnn_qgemm would return.  Host only. */
 typedef enum {
     QNN_KERNEL_TENSOR = 1, QNN_KERNEL_TENSOR_CTA_PAIR = 2, QNN_KERNEL_BYTES_FEW_COLUMNS = 3,

@@ -42,7 +42,7 @@ static qnn_status check_gemm_desc(const qnn_gemm_desc *d, bool has_thr, int *pat
     if (d->w_fmt == QNN_FMT_FIELDS) {
         // packed w-bit weights against 8-bit activation containers: the few-column kernel only
         if (d->a_fmt != QNN_FMT_INT8 || d->path == QNN_PATH_BITSERIAL) return QNN_ERR_UNSUPPORTED;
-        if (!gemv_fields_fits(d, has_thr)) return QNN_ERR_UNSUPPORTED;
+        if (!gemv_fields_dp4a_fits(d) && !gemv_fields_fits(d, has_thr)) return QNN_ERR_UNSUPPORTED;
         if (path_out) *path_out = QNN_PATH_TCGEN05_I8;
         return QNN_OK;
     }
@@ -182,7 +182,11 @@ qnn_status qnn_qgemm(const qnn_gemm_desc *d, const void *W, const void *A, const
     if (!W || !A || !out) return QNN_ERR_INVALID_ARG;
     if (!aligned16(W) || !aligned16(A) || !aligned16(out) || (thr && (reinterpret_cast<uintptr_t>(thr) & 3u)))
         return QNN_ERR_ALIGNMENT;
-    if (d->w_fmt == QNN_FMT_FIELDS) return gemv_fields_launch(d, W, A, thr, out, (cudaStream_t)stream);
+    if (d->w_fmt == QNN_FMT_FIELDS) {
+        // a few columns: byte dot products on the CUDA cores; more: the tensor-core form
+        if (gemv_fields_dp4a_fits(d)) return gemv_fields_dp4a_launch(d, W, A, thr, out, (cudaStream_t)stream);
+        return gemv_fields_launch(d, W, A, thr, out, (cudaStream_t)stream);
+    }
     // 8-bit containers with a handful of columns and no path forced: byte dot products,
     // one warp per weight row (a tensor-core tile would be almost empty)
     if (d->path == QNN_PATH_AUTO && d->w_fmt == QNN_FMT_INT8 && gemv_i8_fits(d))

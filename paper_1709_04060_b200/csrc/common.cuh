@@ -71,6 +71,9 @@ qnn_status gemv_i8_launch(const qnn_gemm_desc *d, const void *W, const void *A,
 bool gemv_planes_fits(const qnn_gemm_desc *d);
 qnn_status gemv_planes_launch(const qnn_gemm_desc *d, const void *W, const void *A,
                               const int32_t *thr, void *out, cudaStream_t s);
+bool gemv_fields_dp4a_fits(const qnn_gemm_desc *d);
+qnn_status gemv_fields_dp4a_launch(const qnn_gemm_desc *d, const void *W, const void *A,
+                                   const int32_t *thr, void *out, cudaStream_t s);
 bool gemv_fields_fits(const qnn_gemm_desc *d, bool has_thr);
 qnn_status gemv_fields_launch(const qnn_gemm_desc *d, const void *W, const void *A,
                               const int32_t *thr, void *out, cudaStream_t s);
