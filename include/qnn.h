@@ -132,7 +132,11 @@ typedef struct {
                              conclusion names; it differs from the exact one by at
                              most K * sum_{i+j<s} 2^(i+j), and the bit-serial kernels
                              skip the AND/POPC work of those pairs.  A BIPOLAR
-                             operand counts as one plane (index 0).               */
+                             operand counts as one plane (index 0).  (Apart from
+                             this, and exactly: the tiled bit-plane kernel skips a
+                             plane pair wherever one of its 64-row x 512-bit plane
+                             tiles holds no set bit -- the bit-level sparsity the
+                             same sentence of the paper names.)                   */
 } qnn_gemm_desc;
 
 /* Scratch bytes qnn_qgemm can use for this problem (0: none).  The workspace is OPTIONAL:

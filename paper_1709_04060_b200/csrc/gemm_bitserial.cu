@@ -10,6 +10,15 @@
 // The popc(A[j]) / popc(W[i]) correction sums are gathered while the tiles are
 // staged into shared memory, so they cost 1/64 of the main loop.
 //
+// Bit-level sparsity (named with the approximate product in the paper's conclusion; this half of
+// it is exact): while a 64 x 512-bit tile of a plane is staged the CTA notes whether it holds any
+// set bit, and the AND/POPC work of a plane pair is skipped for that depth step when either tile
+// is all zero (popc(0 & x) = 0).  Operands whose high-order planes are empty over whole tiles --
+// small activations in a wide container, pruned weight blocks -- then cost only their occupied
+// planes.  The XNOR form of two bipolar operands has no such zero and is never skipped, and
+// kernels with fewer than four plane pairs do not look (the bookkeeping costs 1-2 % of a dense
+// product with 4 to 16 pairs, but 6 % of one with two).
+//
 // Tiling: one CTA (8 warps) per 64 x 64 output tile, depth staged 16 words at a
 // time.  Lanes run along the output-channel dimension (rows m0+lane, m0+32+lane)
 // so that (a) weight words are read conflict-free from a 17-word-pitch tile while
@@ -48,7 +57,9 @@ qgemm_bitserial_kernel(const BsParams p) {
     __shared__ uint32_t Ws[WB][BS_BM][BS_PITCH];
     __shared__ uint32_t As[AB][BS_BN][BS_PITCH];
     __shared__ int corr_s[64];
+    __shared__ unsigned nz_s[2][2];              // [depth step parity][W, A]: planes with a set bit in the staged tile
 
+    constexpr bool SPARSE = WB * AB >= 4 && MODE != BS_BOTH_BIPOLAR;     // look for empty plane tiles
     pdl_wait();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int m0 = blockIdx.y * BS_BM, n0 = blockIdx.x * BS_BN;
@@ -60,6 +71,8 @@ qgemm_bitserial_kernel(const BsParams p) {
 #pragma unroll
         for (int nn = 0; nn < BS_TN; ++nn) acc[t][nn] = 0;
     int corr_part[4] = {0, 0, 0, 0};             // rows lr, lr+16, lr+32, lr+48
+    if (tid < 4) (&nz_s[0][0])[tid] = 0u;
+    __syncthreads();
 
     // implicit convolution: first tap of the four output pixels this thread stages
     int cv_ih0[4], cv_iw0[4];
@@ -75,7 +88,9 @@ qgemm_bitserial_kernel(const BsParams p) {
         }
     }
 
-    for (int kw0 = 0; kw0 < p.kw; kw0 += BS_KT) {
+    for (int kw0 = 0, step = 0; kw0 < p.kw; kw0 += BS_KT, ++step) {
+        const int par = step & 1;
+        unsigned w_nz = 0, a_nz = 0;             // planes of which this thread staged a non-zero word
         const int c = kw0 + lc;
         const bool c_ok = c < p.kw;
         int cv_kh = 0, cv_kw = 0, cv_word = 0;
@@ -93,6 +108,7 @@ qgemm_bitserial_kernel(const BsParams p) {
                 uint32_t v = 0;
                 if (c_ok && m < p.M) v = p.W[((size_t)i * p.M + m) * p.kw + c];
                 Ws[i][r][lc] = v;
+                if (SPARSE) w_nz |= v ? (1u << i) : 0u;
                 if (MODE == BS_A_BIPOLAR) corr_part[q] += p.corr[i] * __popc(v);
             }
 #pragma unroll
@@ -109,38 +125,68 @@ qgemm_bitserial_kernel(const BsParams p) {
                     v = p.A[((size_t)j * p.N + n) * p.kw + c];
                 }
                 As[j][r][lc] = v;
+                if (SPARSE) a_nz |= v ? (1u << j) : 0u;
                 if (MODE == BS_W_BIPOLAR) corr_part[q] += p.corr[j] * __popc(v);
             }
-        __syncthreads();
-
-#pragma unroll 2
-        for (int cc = 0; cc < BS_KT; ++cc) {
-            uint32_t wv[2][WB], av[BS_TN][AB];
-#pragma unroll
-            for (int t = 0; t < 2; ++t)
-#pragma unroll
-                for (int i = 0; i < WB; ++i) wv[t][i] = Ws[i][lane + 32 * t][cc];
-#pragma unroll
-            for (int nn = 0; nn < BS_TN; ++nn)
-#pragma unroll
-                for (int j = 0; j < AB; ++j) av[nn][j] = As[j][warp * BS_TN + nn][cc];
-            // plane pair outermost: a pair that is left out (coefficient 0, uniform) costs one branch
-#pragma unroll
-            for (int i = 0; i < WB; ++i)
-#pragma unroll
-                for (int j = 0; j < AB; ++j) {
-                    const int cf = p.coef[i][j];
-                    if (cf == 0) continue;
-#pragma unroll
-                    for (int nn = 0; nn < BS_TN; ++nn)
-#pragma unroll
-                        for (int t = 0; t < 2; ++t) {
-                            const uint32_t x = (MODE == BS_BOTH_BIPOLAR) ? (wv[t][i] ^ av[nn][j])
-                                                                          : (wv[t][i] & av[nn][j]);
-                            acc[t][nn] += cf * __popc(x);
-                        }
-                }
+        if (SPARSE) {
+            w_nz = __reduce_or_sync(0xffffffffu, w_nz);
+            a_nz = __reduce_or_sync(0xffffffffu, a_nz);
+            if (lane == 0) {
+                if (w_nz) atomicOr(&nz_s[par][0], w_nz);
+                if (a_nz) atomicOr(&nz_s[par][1], a_nz);
+            }
         }
+        __syncthreads();
+        // plane pairs to run in this depth step: coefficient not zero, both tiles occupied
+        unsigned live = 0, wanted = 0;
+#pragma unroll
+        for (int i = 0; i < WB; ++i)
+#pragma unroll
+            for (int j = 0; j < AB; ++j) {
+                if (p.coef[i][j] == 0) continue;
+                wanted |= 1u << (4 * i + j);
+                if (!SPARSE || (((nz_s[par][0] >> i) & 1u) && ((nz_s[par][1] >> j) & 1u)))
+                    live |= 1u << (4 * i + j);
+            }
+        if (SPARSE && tid < 2) nz_s[par ^ 1][tid] = 0u;    // the other parity's flags: last read a step ago, next written a step ahead
+
+        // Two copies of the depth step: when every pair with a coefficient runs (dense operands)
+        // the loop carries no per-pair test, so it costs what it did without the skipping.
+#define QNN_BS_STEP(SKIP_TEST)                                                                         \
+        _Pragma("unroll 2")                                                                            \
+        for (int cc = 0; cc < BS_KT; ++cc) {                                                           \
+            uint32_t wv[2][WB], av[BS_TN][AB];                                                         \
+            _Pragma("unroll")                                                                          \
+            for (int t = 0; t < 2; ++t)                                                                \
+                _Pragma("unroll")                                                                      \
+                for (int i = 0; i < WB; ++i) wv[t][i] = Ws[i][lane + 32 * t][cc];                      \
+            _Pragma("unroll")                                                                          \
+            for (int nn = 0; nn < BS_TN; ++nn)                                                         \
+                _Pragma("unroll")                                                                      \
+                for (int j = 0; j < AB; ++j) av[nn][j] = As[j][warp * BS_TN + nn][cc];                 \
+            /* plane pair outermost: a pair that is left out (uniform) costs one branch */             \
+            _Pragma("unroll")                                                                          \
+            for (int i = 0; i < WB; ++i)                                                               \
+                _Pragma("unroll")                                                                      \
+                for (int j = 0; j < AB; ++j) {                                                         \
+                    const int cf = p.coef[i][j];                                                       \
+                    if (SKIP_TEST) continue;                                                           \
+                    _Pragma("unroll")                                                                  \
+                    for (int nn = 0; nn < BS_TN; ++nn)                                                 \
+                        _Pragma("unroll")                                                              \
+                        for (int t = 0; t < 2; ++t) {                                                  \
+                            const uint32_t x = (MODE == BS_BOTH_BIPOLAR) ? (wv[t][i] ^ av[nn][j])      \
+                                                                          : (wv[t][i] & av[nn][j]);    \
+                            acc[t][nn] += cf * __popc(x);                                              \
+                        }                                                                              \
+                }                                                                                      \
+        }
+        if (!SPARSE || live == wanted) {
+            QNN_BS_STEP(cf == 0)
+        } else {
+            QNN_BS_STEP(!((live >> (4 * i + j)) & 1u))
+        }
+#undef QNN_BS_STEP
         __syncthreads();
     }
 
