@@ -15,10 +15,11 @@
 // results (Section 3.1), thresholds counted as T(x, t) of Section 2.1.1.
 //
 // Against the tensor-core form of the same product (gemv_fields.cu) this kernel has no serial
-// per-SM pipeline to fill, but dp4a issues at only 16 lanes per clock and SM on this GPU (64 byte
-// products per clock and SM: 3.9 us per column at 8192 x 8192), so it is the faster one for a
-// single column (7.7 / 10.3 us against 12.5 / 14.7 us at 8192 x 8192 with 2- / 4-bit fields) and,
-// with 1- or 2-bit fields, for two.
+// per-SM pipeline to fill, but every further column adds its shared-memory reads and dot products
+// to each warp's dependent chain (about 4 us per column at 8192 x 8192; the counters show load
+// latency, global and shared, not a saturated pipe), so it is the faster one for a single column
+// (7.7 / 10.3 us against 12.5 / 14.7 us at 8192 x 8192 with 2- / 4-bit fields) and, with 1- or
+// 2-bit fields, for two.
 #include <stdlib.h>
 
 #include "common.cuh"
