@@ -184,7 +184,7 @@ qnn_status qnn_qgemm(const qnn_gemm_desc *d, const void *W, const void *A,
  *                       tensor-core kernel
  *   BITPLANES operands  N <= 16: one warp per weight row over the planes; else the tiled
  *                       AND/POPC kernel
- *   FIELDS weights      N <= 16 only: one column (two with 1- or 2-bit fields): one warp per
+ *   FIELDS weights      N <= 16 only: one or two columns: one warp per
  *                       packed weight row, an AND and a 4-way byte dot product per word and
  *                       field position; more columns: packed weights expanded inside a
  *                       tensor-core kernel

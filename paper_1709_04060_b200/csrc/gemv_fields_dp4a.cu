@@ -17,9 +17,9 @@
 // Against the tensor-core form of the same product (gemv_fields.cu) this kernel has no serial
 // per-SM pipeline to fill, but every further column adds its shared-memory reads and dot products
 // to each warp's dependent chain (about 4 us per column at 8192 x 8192; the counters show load
-// latency, global and shared, not a saturated pipe), so it is the faster one for a single column
-// (7.7 / 10.3 us against 12.5 / 14.7 us at 8192 x 8192 with 2- / 4-bit fields) and, with 1- or
-// 2-bit fields, for two.
+// latency, global and shared, not a saturated pipe), so it is the faster one for one column
+// (7.0 / 9.4 us against 12.5 / 14.7 us at 8192 x 8192 with 2- / 4-bit fields) and for two
+// (11.2 / 11.7 us against 12.7 / 15.0 us).
 #include <stdlib.h>
 
 #include "common.cuh"
@@ -28,7 +28,7 @@ namespace qnn {
 
 constexpr int FD_THREADS = 256;
 constexpr int FD_COLS = 4;            // most columns per CTA (blockIdx.y picks the block of columns)
-constexpr int FD_MAX_N = 2;           // more columns (4-bit fields: more than one): the tensor-core form
+constexpr int FD_MAX_N = 2;           // more columns: the tensor-core form
 
 struct FdParams {
     const uint8_t *W;      // [M][ldf] packed fields
@@ -44,6 +44,9 @@ struct FdParams {
     int out_bits, out_fmt, ld_out;
 };
 
+// Rows a warp takes at a time: two (measured faster) for 2-bit fields x 1 column and 4-bit fields x 2.
+__host__ __device__ constexpr int fd_rows_at_a_time(int F, int NC) { return (8 / F) * NC == 4 ? 2 : 1; }
+
 template <bool A_SIGNED>
 __device__ __forceinline__ int fd_dot4(uint32_t w, uint32_t a, int c) {
     int d;
@@ -56,9 +59,10 @@ __device__ __forceinline__ int fd_dot4(uint32_t w, uint32_t a, int c) {
 // fewer columns, fewer registers, more warps per SM with loads in flight).  Shared memory:
 // [cols_alloc][col_bytes] columns, then FD_COLS column sums.
 template <int F, bool A_SIGNED, int NC>
-__global__ void __launch_bounds__(FD_THREADS, NC == 1 ? 6 : (NC == 2 ? 5 : 4))
+__global__ void __launch_bounds__(FD_THREADS, 4)
 gemv_fields_dp4a_kernel(const FdParams p) {
     constexpr int S = 8 / F;
+    constexpr int R = fd_rows_at_a_time(F, NC);
     constexpr uint32_t MASK = (F == 1 ? 0x01010101u : (F == 2 ? 0x03030303u : 0x0f0f0f0fu));
     constexpr int GROUP = 32 * S;                 // depth indices per 32 packed bytes
     constexpr int GSTRIDE = GROUP + 32;           // their stride in shared memory
@@ -99,71 +103,88 @@ gemv_fields_dp4a_kernel(const FdParams p) {
     __syncthreads();
 
     const int n_thr = p.thr ? (1 << p.out_bits) - 1 : 0;
-    for (int m = m_first; m < p.M; m += rows_per_grid) {
-        int acc[NC][S];
+    // R rows at a time: their loads are in flight together and they share the reads of the columns
+    for (int m = m_first; m < p.M; m += R * rows_per_grid) {
+        int acc[R][NC][S];
 #pragma unroll
-        for (int c = 0; c < NC; ++c)
+        for (int r = 0; r < R; ++r)
 #pragma unroll
-            for (int s = 0; s < S; ++s) acc[c][s] = 0;
-        const uint4 *wrow = reinterpret_cast<const uint4 *>(p.W + (size_t)m * p.ldf);
+            for (int c = 0; c < NC; ++c)
+#pragma unroll
+                for (int s = 0; s < S; ++s) acc[r][c][s] = 0;
+        const uint4 *wrow[R];
+        bool row_ok[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            row_ok[r] = m + r * rows_per_grid < p.M;
+            wrow[r] = reinterpret_cast<const uint4 *>(p.W + (size_t)(row_ok[r] ? m + r * rows_per_grid : m) * p.ldf);
+        }
 #pragma unroll 4
         for (int q = lane; q < p.steps; q += 32) {
-            const uint4 w = (m == m_first && q == lane) ? w_first : __ldcs(wrow + q);
+            uint4 w[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r) w[r] = (r == 0 && m == m_first && q == lane) ? w_first : __ldcs(wrow[r] + q);
             // 16 packed bytes = one half (q & 1) of group q / 2: field position s of these bytes is
             // depth GROUP * (q / 2) + 32 s + 16 (q & 1) .. + 15
             const uint8_t *a0 = fd_smem + (q >> 1) * GSTRIDE + 16 * (q & 1);
 #pragma unroll
             for (int s = 0; s < S; ++s) {
-                const uint32_t wx = w.x & (MASK << (F * s)), wy = w.y & (MASK << (F * s));
-                const uint32_t wz = w.z & (MASK << (F * s)), ww = w.w & (MASK << (F * s));
 #pragma unroll
                 for (int c = 0; c < NC; ++c) {
                     if (NC == 1 || c < ncols) {
                         const uint4 a = *reinterpret_cast<const uint4 *>(a0 + (size_t)c * p.col_bytes + 32 * s);
-                        acc[c][s] = fd_dot4<A_SIGNED>(wx, a.x, acc[c][s]);
-                        acc[c][s] = fd_dot4<A_SIGNED>(wy, a.y, acc[c][s]);
-                        acc[c][s] = fd_dot4<A_SIGNED>(wz, a.z, acc[c][s]);
-                        acc[c][s] = fd_dot4<A_SIGNED>(ww, a.w, acc[c][s]);
+#pragma unroll
+                        for (int r = 0; r < R; ++r) {
+                            acc[r][c][s] = fd_dot4<A_SIGNED>(w[r].x & (MASK << (F * s)), a.x, acc[r][c][s]);
+                            acc[r][c][s] = fd_dot4<A_SIGNED>(w[r].y & (MASK << (F * s)), a.y, acc[r][c][s]);
+                            acc[r][c][s] = fd_dot4<A_SIGNED>(w[r].z & (MASK << (F * s)), a.z, acc[r][c][s]);
+                            acc[r][c][s] = fd_dot4<A_SIGNED>(w[r].w & (MASK << (F * s)), a.w, acc[r][c][s]);
+                        }
                     }
                 }
             }
         }
-        int tot[NC];
 #pragma unroll
-        for (int c = 0; c < NC; ++c) {
-            tot[c] = 0;
+        for (int r = 0; r < R; ++r) {
+            if (!row_ok[r]) continue;                      // warp-uniform
+            const int mr = m + r * rows_per_grid;
+            int tot[NC];
 #pragma unroll
-            for (int s = 0; s < S; ++s) tot[c] += acc[c][s] >> (F * s);       // exact: a multiple of 2^(F s)
-        }
+            for (int c = 0; c < NC; ++c) {
+                tot[c] = 0;
 #pragma unroll
-        for (int off = 16; off >= 1; off >>= 1)
+                for (int s = 0; s < S; ++s) tot[c] += acc[r][c][s] >> (F * s);       // exact: a multiple of 2^(F s)
+            }
 #pragma unroll
-            for (int c = 0; c < NC; ++c) tot[c] += __shfl_xor_sync(0xffffffffu, tot[c], off);
+            for (int off = 16; off >= 1; off >>= 1)
+#pragma unroll
+                for (int c = 0; c < NC; ++c) tot[c] += __shfl_xor_sync(0xffffffffu, tot[c], off);
 
-        int a = 0;                                         // lane c finishes column n0 + c
+            int a = 0;                                     // lane c finishes column n0 + c
 #pragma unroll
-        for (int c = 0; c < NC; ++c)
-            if (lane == c) a = tot[c];
-        if (lane < ncols) {
-            a = p.w_scale * a + p.w_off * colsum[lane];
-            const int n = n0 + lane;
-            if (!p.thr) {
-                reinterpret_cast<int32_t *>(p.out)[(size_t)n * p.M + m] = a;
-            } else {
-                int code = 0;
-                for (int q = 0; q < n_thr; ++q) code += (a >= __ldg(p.thr + (size_t)m * n_thr + q)) ? 1 : 0;
-                if (p.out_fmt == QNN_FMT_INT8) {
-                    uint8_t *o = reinterpret_cast<uint8_t *>(p.out) + (size_t)n * p.ld_out;
-                    o[m] = (uint8_t)code;
-                    if (m == p.M - 1)                          // the pad bytes of the column
-                        for (int mm = p.M; mm < p.ld_out; ++mm) o[mm] = 0;
+            for (int c = 0; c < NC; ++c)
+                if (lane == c) a = tot[c];
+            if (lane < ncols) {
+                a = p.w_scale * a + p.w_off * colsum[lane];
+                const int n = n0 + lane;
+                if (!p.thr) {
+                    reinterpret_cast<int32_t *>(p.out)[(size_t)n * p.M + mr] = a;
                 } else {
-                    // bit-plane words are shared by 32 rows that other warps own: set single bits
-                    const int mw = (p.M + 31) >> 5;
-                    for (int b = 0; b < p.out_bits; ++b)
-                        if ((code >> b) & 1)
-                            atomicOr(reinterpret_cast<uint32_t *>(p.out) + ((size_t)b * p.N + n) * mw + (m >> 5),
-                                     1u << (m & 31));
+                    int code = 0;
+                    for (int q = 0; q < n_thr; ++q) code += (a >= __ldg(p.thr + (size_t)mr * n_thr + q)) ? 1 : 0;
+                    if (p.out_fmt == QNN_FMT_INT8) {
+                        uint8_t *o = reinterpret_cast<uint8_t *>(p.out) + (size_t)n * p.ld_out;
+                        o[mr] = (uint8_t)code;
+                        if (mr == p.M - 1)                     // the pad bytes of the column
+                            for (int mm = p.M; mm < p.ld_out; ++mm) o[mm] = 0;
+                    } else {
+                        // bit-plane words are shared by 32 rows that other warps own: set single bits
+                        const int mw = (p.M + 31) >> 5;
+                        for (int b = 0; b < p.out_bits; ++b)
+                            if ((code >> b) & 1)
+                                atomicOr(reinterpret_cast<uint32_t *>(p.out) + ((size_t)b * p.N + n) * mw + (mr >> 5),
+                                         1u << (mr & 31));
+                    }
                 }
             }
         }
@@ -191,7 +212,7 @@ static size_t fd_smem_bytes(const qnn_gemm_desc *d, int *col_bytes_out) {
     return (size_t)fd_cols_per_cta(d->N) * (size_t)col_bytes + FD_COLS * sizeof(int);
 }
 
-// One column (two with 1- or 2-bit fields) whose staged form fits shared memory, and accumulators
+// One or two columns whose staged form fits shared memory, and accumulators
 // that cannot overflow (a field position's partial sum is at most 2^8 * |a|max * K).
 // QNN_FIELDS_KERNEL=tensor in the environment keeps the tensor-core form, =dp4a widens this one to
 // 16 columns (tests).
@@ -199,7 +220,7 @@ bool gemv_fields_dp4a_fits(const qnn_gemm_desc *d) {
     if (d->w_fmt != QNN_FMT_FIELDS || d->a_fmt != QNN_FMT_INT8 || d->w_bits > 4) return false;
     const char *force = getenv("QNN_FIELDS_KERNEL");
     if (force && force[0] == 't') return false;
-    const int max_n = (force && force[0] == 'd') ? 16 : (fd_field_bits(d->w_bits) == 4 ? 1 : FD_MAX_N);
+    const int max_n = (force && force[0] == 'd') ? 16 : FD_MAX_N;
     if (d->N > max_n) return false;
     if ((long long)ceil_div(d->K, 32 * (8 / fd_field_bits(d->w_bits))) * (32 * (8 / fd_field_bits(d->w_bits)) + 32) > (48 << 10))
         return false;                                       // a column's staged form: at most 48 KB
@@ -263,7 +284,7 @@ qnn_status gemv_fields_dp4a_launch(const qnn_gemm_desc *d, const void *W, const 
     // then taking row blocks in turn
     int per_sm = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, FD_THREADS, smem) != cudaSuccess || per_sm < 1) per_sm = 1;
-    const int row_blocks = ceil_div(d->M, FD_THREADS / 32);
+    const int row_blocks = ceil_div(ceil_div(d->M, FD_THREADS / 32), fd_rows_at_a_time(F, nc));
     const int max_blocks = sm_count() * per_sm;
     dim3 grid(row_blocks < max_blocks ? row_blocks : max_blocks, ceil_div(d->N, nc));
     void *args[] = {(void *)&p};
