@@ -195,6 +195,7 @@ def test_partial_last_round_is_shared_by_cta_pairs(qb, monkeypatch, M, N, K, w, 
     (480, 11520, 384, 2, 3),     # ragged last channel tile (224 of 256), 1 + 2 k-blocks, bisection epilogue
     (320, 12800, 700, 4, 4),     # second channel tile holds 64 channels: three column groups have no owner
     (768, 8448, 272, 1, 1),      # 99 tiles: 25 split, the second half of the depth is a ragged k-block
+    (512, 11400, 640, 2, 2),     # the last tile of pixels is ragged (136 of 256) and is among the split ones
 ])
 def test_pair_kernel_split_last_round(qb, monkeypatch, M, N, K, w, a):
     """CTA-pair kernel with a workspace: the tiles of a last round that would keep at most half of the
