@@ -368,19 +368,28 @@ def run_b200(args):
     for (w, a) in PAIRS:
         c = synth.gemm_case(2000 + 10 * w + a, DIM, DIM, DIM, w, a)
         Wd = qb.to_device_logical(c.W, c.w_enc)
-        A_host = torch.from_numpy(c.At.astype(np.uint8)).pin_memory()
         prob = {
             "w": w, "a": a, "case": c,
             "Wp": qb.pack(Wd, w, c.w_enc, INT8),
-            "A_host": A_host,
-            "A_log": A_host.cuda(),
+            "A_log": torch.from_numpy(c.At.astype(np.uint8)).cuda(),
             "A_packed": torch.empty(DIM * DIM, dtype=torch.uint8, device="cuda"),
             "thr": torch.from_numpy(c.thr).cuda(),
             "out": torch.empty(DIM * DIM, dtype=torch.uint8, device="cuda"),
-            "out_host": torch.empty(DIM * DIM, dtype=torch.uint8).pin_memory(),
             "pd": qb.qnn_pack_desc(DIM, DIM, a, c.a_enc, INT8),
             "gd": qb.gemm_desc(DIM, DIM, DIM, w, a, a, c.w_enc, c.a_enc, INT8, INT8),
         }
+        # End-to-end leg: few-bit data crosses the host link packed.  The activations wait in pinned
+        # host memory as bit planes (a bits per element; packed once, at set-up, by the library's
+        # packer), are widened to 8-bit containers on the device, and the output codes go back as
+        # bit planes (a bits per code).
+        PL = qb.QNN_FMT_BITPLANES
+        planes_dev = qb.pack(prob["A_log"], a, c.a_enc, PL)
+        prob["rd"] = qb.qnn_pack_desc(DIM, DIM, a, c.a_enc, PL)
+        prob["A_planes"] = planes_dev
+        prob["A_planes_host"] = planes_dev.cpu().pin_memory()
+        prob["gd_pl"] = qb.gemm_desc(DIM, DIM, DIM, w, a, a, c.w_enc, c.a_enc, INT8, PL)
+        prob["out_pl"] = torch.empty(qb.qnn_gemm_out_bytes(prob["gd_pl"], True), dtype=torch.uint8, device="cuda")
+        prob["out_pl_host"] = torch.empty(prob["out_pl"].numel(), dtype=torch.uint8).pin_memory()
         del Wd
         problems.append(prob)
     # scratch the library may use to split a half-empty last round of tiles between SM pairs (its
@@ -394,6 +403,7 @@ def run_b200(args):
     # problem i (tensor bound) runs on the main one; events order each GEMM after its packer
     # and each packer after the GEMM that last read its output buffer.
     s_pack = torch.cuda.Stream() if args.overlap else None
+    s_out = torch.cuda.Stream()
 
     def step(gemm_events=None, host_io=False):
         main = torch.cuda.current_stream()
@@ -405,18 +415,24 @@ def run_b200(args):
                     s_pack.wait_event(p["gemm_done"])
                 with torch.cuda.stream(s_pack):
                     if host_io:
-                        p["A_log"].copy_(p["A_host"], non_blocking=True)
-                    qb.check(qb.qnn_pack(p["pd"], p["A_log"], p["A_packed"]))
+                        p["A_planes"].copy_(p["A_planes_host"], non_blocking=True)
+                        qb.check(qb.qnn_planes_to_int8(p["rd"], p["A_planes"], p["A_packed"]))
+                    else:
+                        qb.check(qb.qnn_pack(p["pd"], p["A_log"], p["A_packed"]))
                     p["packed"] = torch.cuda.Event()
                     p["packed"].record(s_pack)
                 main.wait_event(p["packed"])
+            elif host_io:
+                p["A_planes"].copy_(p["A_planes_host"], non_blocking=True)
+                qb.check(qb.qnn_planes_to_int8(p["rd"], p["A_planes"], p["A_packed"]))
             else:
-                if host_io:
-                    p["A_log"].copy_(p["A_host"], non_blocking=True)
                 qb.check(qb.qnn_pack(p["pd"], p["A_log"], p["A_packed"]))
             if gemm_events is not None:
                 e0 = torch.cuda.Event(enable_timing=True); e0.record()
-            qb.check(qb.qnn_qgemm(p["gd"], p["Wp"], p["A_packed"], p["thr"], p["out"], gemm_ws, gemm_ws.numel()))
+            if host_io:
+                qb.check(qb.qnn_qgemm(p["gd_pl"], p["Wp"], p["A_packed"], p["thr"], p["out_pl"], gemm_ws, gemm_ws.numel()))
+            else:
+                qb.check(qb.qnn_qgemm(p["gd"], p["Wp"], p["A_packed"], p["thr"], p["out"], gemm_ws, gemm_ws.numel()))
             if gemm_events is not None:
                 e1 = torch.cuda.Event(enable_timing=True); e1.record()
                 gemm_events.append((e0, e1))
@@ -424,7 +440,12 @@ def run_b200(args):
                 p["gemm_done"] = torch.cuda.Event()
                 p["gemm_done"].record(main)
             if host_io:
-                p["out_host"].copy_(p["out"], non_blocking=True)
+                # the read-back runs on its own stream, so that the next GEMM does not queue behind it
+                s_out.wait_stream(main)
+                with torch.cuda.stream(s_out):
+                    p["out_pl_host"].copy_(p["out_pl"], non_blocking=True)
+        if host_io:
+            main.wait_stream(s_out)
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -535,8 +556,11 @@ def run_b200(args):
                    "gops_paper_convention": 2 * value / 1e9},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT,
-                "h2d_bytes_per_step": len(PAIRS) * DIM * DIM, "d2h_bytes_per_step": len(PAIRS) * DIM * DIM,
-                "steps": e2e_steps},
+                "h2d_bytes_per_step": int(sum(p["A_planes_host"].numel() for p in problems)),
+                "d2h_bytes_per_step": int(sum(p["out_pl_host"].numel() for p in problems)),
+                "steps": e2e_steps,
+                "note": "activations cross the host link as bit planes (a bits per element) and are widened to "
+                        "8-bit containers on the device; output codes return as bit planes"},
         "gpu_launches": int(launches),
         "roofline": roofline_entry(achieved_tops, gemm_avg_ms, ms * 1e-3, clocks, peaks, measured),
         "per_pair_tmacs": per_pair,

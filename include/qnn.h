@@ -111,6 +111,14 @@ size_t qnn_packed_bytes(const qnn_pack_desc *d);
  * full, padding included.  Both 16-byte aligned. */
 qnn_status qnn_pack(const qnn_pack_desc *d, const void *logical, void *packed, void *stream);
 
+/* A BITPLANES operand widened to INT8 containers of the same values (Section 3.1's planes to
+ * Section 3's 8-bit operands): d describes the source (d->fmt must be QNN_FMT_BITPLANES; rows, K,
+ * bits, enc); planes: uint32 [bits][rows][ceil(K/32)]; containers: [rows][K rounded up to 16],
+ * written in full, pad bytes zero.  For data that is stored or shipped packed -- `bits` instead of
+ * 8 bits per element over the host link -- and multiplied on the tensor cores.  Both pointers
+ * 16-byte aligned. */
+qnn_status qnn_planes_to_int8(const qnn_pack_desc *d, const void *planes, void *containers, void *stream);
+
 /* ---- fused GEMM + threshold (Sections 3.1 and 2.1.1) ---------------------- */
 
 typedef struct {

@@ -32,7 +32,7 @@ QNN_FMT_BITPLANES, QNN_FMT_INT8, QNN_FMT_FIELDS = 0, 1, 2
 QNN_PATH_AUTO, QNN_PATH_BITSERIAL, QNN_PATH_TCGEN05_I8 = 0, 1, 2
 
 EXPORTS = (
-    "qnn_packed_ld", "qnn_packed_bytes", "qnn_pack", "qnn_gemm_workspace_bytes",
+    "qnn_packed_ld", "qnn_packed_bytes", "qnn_pack", "qnn_planes_to_int8", "qnn_gemm_workspace_bytes",
     "qnn_gemm_out_bytes", "qnn_qgemm", "qnn_qgemm_kernel", "qnn_conv_out_h", "qnn_conv_out_w",
     "qnn_conv_lowered_k", "qnn_conv_lowered_bytes", "qnn_conv_workspace_bytes",
     "qnn_conv_out_bytes", "qnn_im2col", "qnn_qconv", "qnn_qconv_static", "qnn_maxpool",
@@ -74,6 +74,8 @@ _lib.qnn_packed_bytes.restype = _sz
 _lib.qnn_packed_bytes.argtypes = [_P(qnn_pack_desc)]
 _lib.qnn_pack.restype = _ci
 _lib.qnn_pack.argtypes = [_P(qnn_pack_desc), _vp, _vp, _vp]
+_lib.qnn_planes_to_int8.argtypes = [_P(qnn_pack_desc), _vp, _vp, _vp]
+_lib.qnn_planes_to_int8.restype = _ci
 _lib.qnn_gemm_workspace_bytes.restype = _sz
 _lib.qnn_gemm_workspace_bytes.argtypes = [_P(qnn_gemm_desc)]
 _lib.qnn_gemm_out_bytes.restype = _sz
@@ -170,6 +172,10 @@ def qnn_packed_bytes(d: qnn_pack_desc) -> int:
 
 def qnn_pack(d, logical, packed, stream=None) -> int:
     return _lib.qnn_pack(ctypes.byref(d), _ptr(logical), _ptr(packed), _stream(stream))
+
+
+def qnn_planes_to_int8(d, planes, containers, stream=None) -> int:
+    return _lib.qnn_planes_to_int8(ctypes.byref(d), _ptr(planes), _ptr(containers), _stream(stream))
 
 
 def qnn_gemm_workspace_bytes(d) -> int:

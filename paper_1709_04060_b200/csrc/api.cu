@@ -147,6 +147,15 @@ qnn_status qnn_pack(const qnn_pack_desc *d, const void *logical, void *packed, v
     return pack_launch(d, logical, packed, (cudaStream_t)stream);
 }
 
+qnn_status qnn_planes_to_int8(const qnn_pack_desc *d, const void *planes, void *containers, void *stream) {
+    if (!d || !planes || !containers) return QNN_ERR_INVALID_ARG;
+    if (d->rows <= 0 || d->K <= 0 || d->bits < 1 || d->bits > 8) return QNN_ERR_INVALID_ARG;
+    if (d->fmt != QNN_FMT_BITPLANES || d->enc < 0 || d->enc > 2) return QNN_ERR_INVALID_ARG;
+    if (!valid_enc(d->enc, d->bits)) return QNN_ERR_UNSUPPORTED;
+    if (!aligned16(planes) || !aligned16(containers)) return QNN_ERR_ALIGNMENT;
+    return planes_to_int8_launch(d, planes, containers, (cudaStream_t)stream);
+}
+
 size_t qnn_gemm_workspace_bytes(const qnn_gemm_desc *d) {
     int path = 0;
     if (check_gemm_desc(d, true, &path) != QNN_OK) return 0;

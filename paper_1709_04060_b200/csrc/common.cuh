@@ -61,6 +61,7 @@ int sm_count();
 
 // Path implementations (one translation unit each).
 qnn_status pack_launch(const qnn_pack_desc *d, const void *logical, void *packed, cudaStream_t s);
+qnn_status planes_to_int8_launch(const qnn_pack_desc *d, const void *planes, void *packed, cudaStream_t s);
 qnn_status gemm_bitserial_launch(const qnn_gemm_desc *d, const void *W, const void *A,
                                  const int32_t *thr, void *out, cudaStream_t s);
 qnn_status gemm_bitserial_conv_launch(const qnn_conv_desc *cv, const qnn_gemm_desc *g, const void *W,

@@ -1,6 +1,7 @@
 // Operand packer: logical bytes -> bit planes (Section 3.1: plane i = bit i of
 // every element, packed along the depth) or zero-padded 8-bit containers
-// (Section 3: operands cast to 8-bit integers).  Also the threshold validator.
+// (Section 3: operands cast to 8-bit integers); bit planes -> 8-bit containers (few-bit data
+// crosses the host link packed and is widened on the device).  Also the threshold validator.
 #include "common.cuh"
 
 namespace qnn {
@@ -71,6 +72,42 @@ __device__ __forceinline__ uint32_t container4(uint32_t x, int bits, int enc) {
     // 2^(8-bits) - 1 fills bits [bits, 8) and cannot carry into the next byte
     const uint32_t sign = low & (0x01010101u << (bits - 1));
     return low | ((sign << 1) * ((1u << (8 - bits)) - 1u));
+}
+
+// Bit planes -> 8-bit containers: one thread per 16 output bytes (16 consecutive depth indices,
+// one half of a plane word).  Four bits of a plane become four bytes by one multiplication
+// (bit b of the nibble lands in bit 0 of byte b); plane i adds them shifted by i.
+__global__ void __launch_bounds__(256) planes_to_int8_kernel(const uint32_t *__restrict__ planes,
+                                                             uint4 *__restrict__ packed, int rows, int K,
+                                                             int kw, int chunks, int bits, int enc) {
+    const long long total = (long long)rows * chunks;
+    for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int r = (int)(idx / chunks), c = (int)(idx - (long long)r * chunks);
+        const int k0 = 16 * c, word = k0 >> 5, shift = k0 & 31;
+        uint32_t o[4] = {0u, 0u, 0u, 0u};
+        for (int i = 0; i < bits; ++i) {
+            const uint32_t x = (planes[((size_t)i * rows + r) * kw + word] >> shift) & 0xFFFFu;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t spread = (((x >> (4 * q)) & 0xFu) * 0x00204081u) & 0x01010101u;
+                // SIGNED: the top plane is the sign, which also fills the container's upper bits
+                const uint32_t mul = (enc == QNN_ENC_SIGNED && i == bits - 1) ? ((0xFFu << i) & 0xFFu) : (1u << i);
+                o[q] |= spread * mul;
+            }
+        }
+        if (enc == QNN_ENC_BIPOLAR) {
+            // bit 1 -> +1, bit 0 -> -1; pad bytes past K stay zero
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                uint32_t v = 0xFFFFFFFFu ^ (o[q] * 0xFEu);
+                const int left = K - (k0 + 4 * q);                 // elements of this word inside the row
+                if (left < 4) v &= left <= 0 ? 0u : (0xFFFFFFFFu >> (8 * (4 - left)));
+                o[q] = v;
+            }
+        }
+        packed[idx] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
 }
 
 // K a multiple of 16 (no padding): one thread per 16 bytes, 16-byte loads and stores.
@@ -147,6 +184,18 @@ __global__ void pack_fields_kernel(const uint8_t *__restrict__ logical, uint32_t
             word |= u << (8 * b + f * s);
         }
     packed[idx] = word;
+}
+
+qnn_status planes_to_int8_launch(const qnn_pack_desc *d, const void *planes, void *packed, cudaStream_t s) {
+    const int threads = 256;
+    const int kw = ceil_div(d->K, 32), chunks = round_up(d->K, 16) / 16;
+    const long long total = (long long)d->rows * chunks;
+    const long long want = (total + threads - 1) / threads, cap = (long long)sm_count() * 16;
+    planes_to_int8_kernel<<<(unsigned)(want < cap ? want : cap), threads, 0, s>>>(
+        (const uint32_t *)planes, (uint4 *)packed, d->rows, d->K, kw, chunks,
+        d->enc == QNN_ENC_BIPOLAR ? 1 : d->bits, d->enc);
+    count_launch();
+    return launch_status();
 }
 
 qnn_status pack_launch(const qnn_pack_desc *d, const void *logical, void *packed, cudaStream_t s) {
