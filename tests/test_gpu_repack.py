@@ -50,3 +50,23 @@ def test_arguments_are_checked_before_launch(qb):
     assert qb.qnn_planes_to_int8(qb.qnn_pack_desc(4, 64, 2, 0, BITPLANES), buf[4:], buf) == qb.QNN_ERR_ALIGNMENT
     assert qb.qnn_planes_to_int8(qb.qnn_pack_desc(0, 64, 2, 0, BITPLANES), buf, buf) == qb.QNN_ERR_INVALID_ARG
     assert qb.qnn_launch_count() == n0
+
+
+@pytest.mark.parametrize("w,a", [(1, 2), (2, 1), (3, 3), (4, 4)])
+def test_packed_in_packed_out_pipeline(qb, w, a):
+    """The benchmark's end-to-end leg at a size the oracle finishes: activations packed as bit planes
+    on the host (the tests' own packer), widened on the device, multiplied on the tensor cores with
+    the threshold epilogue writing bit planes, unpacked on the host: every code against the oracle."""
+    from oracle import oracle as orc
+    from qnn_testutil import decode_out
+    M, N, K = 300, 700, 1100
+    case = synth.gemm_case(9100 + 10 * w + a, M, N, K, w, a)
+    planes = torch.from_numpy(host_pack_planes(case.At, 1 if case.a_enc == synth.BIPOLAR else a, case.a_enc)).cuda()
+    containers = torch.empty(N * round_up(K, 16), dtype=torch.uint8, device="cuda")
+    qb.check(qb.qnn_planes_to_int8(qb.qnn_pack_desc(N, K, a, case.a_enc, BITPLANES), planes, containers))
+    Wp = qb.pack(qb.to_device_logical(case.W, case.w_enc), w, case.w_enc, INT8)
+    d = qb.gemm_desc(M, N, K, w, a, case.out_bits, case.w_enc, case.a_enc, INT8, BITPLANES)
+    out = qb.qgemm(d, Wp, containers, torch.from_numpy(case.thr).cuda())
+    torch.cuda.synchronize()
+    got = decode_out(out.cpu().numpy().view(np.uint8).reshape(-1), BITPLANES, case.out_bits, N, M, False)
+    assert np.array_equal(got, orc.qgemm(case.W, case.At, case.thr).T)
